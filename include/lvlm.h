@@ -1,0 +1,219 @@
+/*
+ * lvlm.h - C ABI of the LightVLM token-reduction / KV-cache-compression kernels (sm_100a).
+ *
+ * The library implements the computation that LightVLM adds to a vision-language model:
+ * pyramid token merging during encoding (paper Section 3.2.1) and KV-cache compression
+ * followed by decoding over the shortened cache (Section 3.2.2), with the settings of
+ * Appendix A.2.  It does not contain a model: callers hand in the tensors of one layer.
+ *
+ * Conventions for every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library never
+ *     allocates, frees or keeps a pointer after the call returns.  `lvlm_dims` itself is a
+ *     HOST struct, read during the call only.
+ *   - Scratch memory comes from the caller: `ws` (device, 256-byte aligned) of at least
+ *     `lvlm_workspace_bytes(op, dims)` bytes.  Its contents need not be preserved or zeroed.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream) and the call returns without synchronising.  Calls that share `ws` or
+ *     any in/out tensor must be ordered by the caller (same stream is enough).
+ *   - Activations are bf16, scores fp32, indices int32.  The innermost dimension of every
+ *     tensor is contiguous and 16-byte aligned.  Only D == 128 is supported.
+ *   - A host-detectable error returns a non-zero `lvlm_status` and enqueues nothing.
+ *     Conditions only the device can see (non-finite score, length beyond capacity) OR a
+ *     `LVLM_DEV_*` bit into `*dev_status` (optional, caller-owned int32 on the device,
+ *     never cleared by the library); the offending access is skipped and the kernel ends
+ *     normally.  No kernel traps or asserts.
+ *   - Results are bit-reproducible from run to run: no floating-point atomics are used.
+ */
+#ifndef LVLM_H_
+#define LVLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LVLM_OK = 0,
+    LVLM_ERR_INVALID_ARG = 1,   /* NULL required pointer, size or range out of bounds */
+    LVLM_ERR_UNSUPPORTED = 2,   /* D != 128, n or cache length beyond the built limits */
+    LVLM_ERR_ALIGNMENT = 3,     /* pointer or stride not 16-byte aligned */
+    LVLM_ERR_WORKSPACE = 4,     /* ws NULL, misaligned or smaller than lvlm_workspace_bytes */
+    LVLM_ERR_CUDA = 5           /* a CUDA runtime call failed (launch, attribute, driver entry) */
+} lvlm_status;
+
+/* bits OR-ed into *dev_status by kernels */
+enum { LVLM_DEV_NONFINITE = 1, LVLM_DEV_TIMEOUT = 2, LVLM_DEV_BOUNDS = 4 };
+
+/* How the r+1 least important image tokens become one token (Section 3.2.1, paragraph 4).
+ * p = 0 is the most important merged token; weights are divided by their sum.
+ *   LINEAR_RANK   the stated weight list W_v = {r+1, r, ..., 1}                 (default)
+ *   GEOMETRIC     (1/2, 1/4, ..., 2^-r, 2^-r): the literal result of repeatedly merging the
+ *                 last two tokens of the queue with equal weights
+ *   UNIFORM       1/(r+1) each
+ *   CUSTOM        caller-supplied list w_custom[0..r]
+ *   NEAREST_KEPT  not in the paper: each dropped token is averaged into the kept token with
+ *                 the highest cosine similarity (lower index wins ties); no extra token */
+typedef enum {
+    LVLM_W_LINEAR_RANK = 0, LVLM_W_GEOMETRIC = 1, LVLM_W_UNIFORM = 2,
+    LVLM_W_CUSTOM = 3, LVLM_W_NEAREST_KEPT = 4
+} lvlm_merge_mode;
+
+typedef enum {
+    LVLM_OP_SCORE_TOKENS = 0, LVLM_OP_SELECT_TOPK = 1, LVLM_OP_MERGE_COMPACT = 2,
+    LVLM_OP_KV_COMPRESS = 3, LVLM_OP_DECODE_ATTN = 4
+} lvlm_op;
+
+/* Problem sizes.  Each entry point lists the fields it reads; the others are ignored.
+ * Strides are in ELEMENTS; 0 selects the packed default given beside the tensor. */
+typedef struct lvlm_dims {
+    int32_t B;        /* sequences in the batch */
+    int32_t H;        /* query heads */
+    int32_t Hkv;      /* key/value heads; H % Hkv == 0; query head h uses KV head h / (H/Hkv) */
+    int32_t D;        /* head dimension (128) */
+    int32_t N;        /* tokens per sequence before the call */
+    int32_t C;        /* hidden channels, a multiple of 8 */
+    int32_t cap;      /* rows allocated per (sequence, KV head) in a K or V cache */
+    int32_t i0;       /* index of the first image token */
+    int32_t n;        /* number of image tokens: the span is [i0, i0+n) */
+    int32_t k;        /* image tokens kept intact (P_unmerged); the other n-k are merged */
+    int32_t q_lo;     /* scoring: first query row (sequence position) of the window */
+    int32_t q_hi;     /* scoring: one past the last query row of the window */
+    int32_t causal;   /* scoring: 1 = row at position p sees keys j <= p; 0 = sees all N keys */
+    int32_t recent;   /* kv_compress: this many newest entries of every head are never evicted */
+    int64_t q_stride_b, q_stride_n, q_stride_h;  /* Q[b][i][h][D]; default packed [B][q_hi-q_lo][H][D] */
+    int64_t kv_stride_b, kv_stride_h;            /* K,V[b][g][row][D], rows packed; default [B][Hkv][cap][D] */
+    int64_t hid_stride_b;                        /* hidden[b][row][C], rows packed; default N*C */
+    int64_t out_stride_b;                        /* hidden_out[b][row][C]; default (rows after the call)*C */
+} lvlm_dims;
+
+/* Library version string (static storage). */
+const char* lvlm_version(void);
+
+/* Text for a status code (static storage). */
+const char* lvlm_status_string(lvlm_status s);
+
+/* Bytes of device scratch `op` needs for `d` (0 if `d` is invalid for that op).  Host only. */
+size_t lvlm_workspace_bytes(int op, const lvlm_dims* d);
+
+/*
+ * Importance of every image token: the attention it receives, summed over the query rows
+ * of a window and averaged over heads (Section 3.2.1, paragraph 3: the per-key "cumsum
+ * attention scores" A, "averaged ... across different heads").
+ *
+ *   s_head[b,h,j] = sum_{p in [q_lo,q_hi)} softmax_over_visible_keys(q[b,p,h] . K[b,h/G] * scale)[j]
+ *   score[b,j-i0]          = (1/H) sum_h s_head[b,h,j]                     j in [i0, i0+n)
+ *   score_head[b,g,j-i0]   = sum_{h in group g} s_head[b,h,j]   (what per-head KV compression uses)
+ *
+ * The softmax of row p is taken over ALL keys it can see (j <= p if d->causal, else all N),
+ * not only over image keys.  The window [0,N) gives the column sums of the full causal
+ * attention matrix; the window [i0+n, N) gives the attention of the instruction text only.
+ *   Q          [B][q_hi-q_lo][H][D] bf16, row 0 = sequence position q_lo (strides d->q_stride_*)
+ *   K          [B][Hkv][cap][D] bf16, rows 0..N-1 valid (strides d->kv_stride_*)
+ *   lse        optional [B][H][q_hi-q_lo] fp32: natural-log sum-exp of each row's scaled
+ *              logits as produced by the attention kernel that ran before; NULL = computed here
+ *   score      [B][n] fp32 out;  score_head optional [B][Hkv][n] fp32 out
+ * Reads d: B,H,Hkv,D,N,cap,i0,n,q_lo,q_hi,causal,q_stride_*,kv_stride_*.
+ * Errors: INVALID_ARG (NULL Q/K/score, i0+n>N, q_lo>=q_hi, q_hi>N, N>cap, H%Hkv), UNSUPPORTED
+ * (D!=128), ALIGNMENT, WORKSPACE.  A non-finite score sets LVLM_DEV_NONFINITE.
+ */
+lvlm_status lvlm_score_tokens(const void* Q, const void* K, const float* lse,
+                              const lvlm_dims* d, float scale,
+                              float* score, float* score_head,
+                              void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Split of the image tokens into P_unmerged and P_merged (Section 3.2.1, paragraph 4): the
+ * total order of the n tokens by (score descending, index ascending).
+ *   score     [B] rows of n fp32, row stride score_stride elements (0 = n)
+ *   rank      [B][n] int32 out: position of token j in the order.  rank < k: kept intact;
+ *             rank >= k: merged, and rank - k is its place in the merge queue
+ *   kept_idx  optional [B][k] int32 out: the kept tokens, ascending
+ *   near_tie  optional [B] int32 out: neighbours (p, p+1) of the order with p+1 >= k whose
+ *             fp32 gap satisfies (s_p - s_{p+1}) < 1e-4 * |s_p|  (ties the caller may report)
+ * -0 equals +0; NaN sorts last and sets LVLM_DEV_NONFINITE (so does an infinity).
+ * Errors: INVALID_ARG (NULL score/rank, B<=0, n<=0, k outside [0,n]), UNSUPPORTED (n > 16384).
+ */
+lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_stride, int k,
+                             int32_t* rank, int32_t* kept_idx, int32_t* near_tie,
+                             void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Merge and compaction (Section 3.2.1, paragraph 4): P_new = W_v x P_merged and
+ * P_compressed = [P_unmerged, P_new], written inside the full sequence:
+ *     [ tokens before the image | kept image tokens, original order | P_new | tokens after ]
+ * With r = n-k-1 the sequence shrinks from N to N-r rows; r <= 0 (k >= n-1) leaves every
+ * tensor unchanged.  In mode NEAREST_KEPT there is no P_new row and the result has
+ * N-(n-k) rows.
+ *   hidden      [B][N][C] bf16 (batch stride d->hid_stride_b)
+ *   hidden_out  [B][rows after][C] bf16, or NULL to compact `hidden` in place
+ *   Kc, Vc      optional [B][Hkv][cap][D] bf16: this layer's keys and values, rows 0..N-1
+ *               valid; compacted IN PLACE with the same map, the merged row being the same
+ *               weighted mean per KV head (pass both or neither)
+ *   pos_ids     optional [B][N] int32, compacted in place; P_new takes the id of the most
+ *               important merged token
+ *   rank        [B][n] int32 from lvlm_select_topk (must be a permutation of 0..n-1)
+ *   w_custom    [n-k] fp32 (device) when mode == CUSTOM, else NULL
+ *   mass        NEAREST_KEPT only, optional [B][N] fp32 in/out: token masses (NULL = all 1)
+ *   new_len     optional [B] int32 out: rows after the call
+ * Reads d: B,N,C,Hkv,D,cap,i0,n,k,hid_stride_b,out_stride_b,kv_stride_*.
+ * Errors: INVALID_ARG (NULL hidden/rank, i0+n>N, k outside [0,n], N>cap with Kc, only one of
+ * Kc/Vc, CUSTOM without w_custom, C%8), UNSUPPORTED (D!=128 with Kc), ALIGNMENT, WORKSPACE.
+ */
+lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* Kc, void* Vc,
+                               int32_t* pos_ids, const int32_t* rank, const lvlm_dims* d,
+                               lvlm_merge_mode mode, const float* w_custom, float* mass,
+                               int32_t* new_len,
+                               void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * KV-cache compression (Section 3.2.2, paragraph 2; Appendix A.2: threshold beta = 0.995,
+ * layers after Layer 5), independently per (sequence, KV head): among the evictable entries
+ *     E = [e_lo[b], min(e_hi[b], len - d->recent))
+ * sort by (acc_score descending, index ascending), keep the shortest prefix whose cumulative
+ * score reaches beta * (total score of E) - the entry that crosses the threshold is kept -
+ * but at most budget - (entries outside E); drop the rest of E.  Survivors keep their order;
+ * K, V, acc_score and pos are compacted in place and len is updated.
+ * The count is exact: scores are taken in integer units of 2^-24 and beta in parts per
+ * million; beta >= 1 disables the threshold (keep all, subject to the budget).
+ *   Kc, Vc     [B][Hkv][cap][D] bf16 in/out        acc_score [B][Hkv][cap] fp32 in/out
+ *   pos        optional [B][Hkv][cap] int32 in/out len [B][Hkv] int32 in/out
+ *   e_lo,e_hi  optional [B] int32 (both or neither); NULL = every entry is evictable
+ *   budget     maximum entries per head after the call; <= 0 means no budget
+ * The paper's use: e = the image span, beta = 0.995, no budget, once before generation.
+ * Periodic use during decoding: e = NULL, beta = 1, budget, d->recent protecting new entries.
+ * Reads d: B,Hkv,D,cap,recent,kv_stride_*.
+ * Errors: INVALID_ARG (NULL Kc/Vc/acc_score/len, beta outside (0,1], one of e_lo/e_hi),
+ * UNSUPPORTED (D!=128, cap > 16384), ALIGNMENT, WORKSPACE.  len > cap sets LVLM_DEV_BOUNDS
+ * and that head is left untouched.
+ */
+lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, int32_t* pos, int32_t* len,
+                             const int32_t* e_lo, const int32_t* e_hi, const lvlm_dims* d,
+                             float beta, int budget,
+                             void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * One decoding step of attention over the (ragged, compressed) cache (Section 3.2.2,
+ * paragraph 1: the current token attends to every cached key and value).
+ *   o[b,h,:] = softmax(q[b,h,:] . K[b,g,0:len[b,g],:]^T * scale) V[b,g,0:len[b,g],:],  g = h/(H/Hkv)
+ *   q        [B][H][D] bf16            out [B][H][D] bf16
+ *   Kc, Vc   [B][Hkv][cap][D] bf16     len [B][Hkv] int32
+ *   k_new, v_new  optional [B][Hkv][D] bf16 (both or neither): appended at row len before
+ *            attending, len += 1.  If len == cap the append is skipped, len stays and
+ *            LVLM_DEV_BOUNDS is set.
+ *   acc_score optional [B][Hkv][cap] fp32 in/out: entry j receives the probabilities of the
+ *            group's query heads, acc_score[b,g,j] += sum_{h in g} p[b,h,j]
+ * A head with len == 0 (and no append) outputs zeros.
+ * Reads d: B,H,Hkv,D,cap,kv_stride_*.
+ * Errors: INVALID_ARG, UNSUPPORTED (D!=128, H/Hkv > 8), ALIGNMENT, WORKSPACE.
+ */
+lvlm_status lvlm_decode_attn(const void* q, void* Kc, void* Vc, int32_t* len,
+                             const void* k_new, const void* v_new, float* acc_score,
+                             const lvlm_dims* d, float scale, void* out,
+                             void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LVLM_H_ */

@@ -375,7 +375,7 @@ def decode_attn(q, Kc, Vc, length, k_new=None, v_new=None, acc_score=None, scale
     [B, Hkv, D] are given they are appended at row len first and len grows by one.
     o[b,h] = softmax(q[b,h] . K[b,g,0:len]^T * scale) V[b,g,0:len],  g = h // G.
     acc_score [B, Hkv, cap] (optional) receives, per cached entry, the probabilities
-    summed over the query heads of the group.
+    summed over the query heads of the group; an appended entry starts from zero.
     Returns dict(out [B,H,D] bf16-rounded float32, Kc, Vc, len, acc_score).
     """
     q = np.asarray(q, dtype=np.float64)
@@ -395,6 +395,8 @@ def decode_attn(q, Kc, Vc, length, k_new=None, v_new=None, acc_score=None, scale
             if k_new is not None:
                 Kc[b, g, ln] = np.asarray(k_new[b, g], dtype=np.float32)
                 Vc[b, g, ln] = np.asarray(v_new[b, g], dtype=np.float32)
+                if acc is not None:
+                    acc[b, g, ln] = 0.0                    # a new entry starts with no score
                 ln += 1
                 length[b, g] = ln
             Kd = Kc[b, g, :ln].astype(np.float64)

@@ -1,0 +1,88 @@
+// Shared helpers of the lvlm kernels: argument checks, bf16 packing, order-preserving keys.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lvlm.h"
+
+namespace lvlm {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxSortN = 16384;      // one CTA ranks at most this many 64-bit keys in shared memory
+constexpr int kMaxGroup = 8;          // query heads per KV head supported by decode attention
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+#define LVLM_RETURN_IF_CUDA(expr)                      \
+    do {                                               \
+        cudaError_t e__ = (expr);                      \
+        if (e__ != cudaSuccess) return LVLM_ERR_CUDA;  \
+    } while (0)
+
+inline lvlm_status launch_status() {
+    return cudaGetLastError() == cudaSuccess ? LVLM_OK : LVLM_ERR_CUDA;
+}
+
+// ---- bf16 <-> fp32 on packed words -------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ---- total order used by selection and eviction --------------------------------------
+// Ascending order of the returned 32-bit value == DESCENDING order of the score; NaN maps to
+// the largest value (sorted last); -0 and +0 map to the same value.
+__device__ __forceinline__ uint32_t desc_key(float s, bool* nonfinite) {
+    uint32_t u = __float_as_uint(s);
+    if ((u & 0x7F800000u) == 0x7F800000u) *nonfinite = true;
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0xFFFFFFFFu;      // NaN
+    if (u == 0x80000000u) u = 0;                                  // -0 -> +0
+    uint32_t asc = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ~asc;
+}
+
+// ---- small block-level primitives ----------------------------------------------------
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Exclusive prefix sum of one int per thread over the block (blockDim.x <= 1024, a multiple
+// of 32).  `scratch` holds 33 ints of shared memory.  Returns the exclusive prefix; *total
+// receives the block sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* scratch, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();                      // scratch may still be read from a previous call
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < nwarp ? scratch[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        scratch[lane] = wi - w;           // exclusive warp offsets
+        if (lane == 31) scratch[32] = wi;
+    }
+    __syncthreads();
+    *total = scratch[32];
+    return scratch[warp] + incl - v;
+}
+
+}  // namespace lvlm
