@@ -103,9 +103,10 @@ def score_tokens(Q, K, q_lo, q_hi, i0, n, causal=True, scale=None):
 def _descending_order(score_row):
     """Indices sorted by (score descending, index ascending); NaN last; -0 == +0."""
     s = np.asarray(score_row, dtype=np.float32).astype(np.float64)
-    s = np.where(np.isnan(s), -np.inf, s)
-    # numpy's stable sort keeps equal keys in index order
-    return np.argsort(-s, kind="stable")
+    nan = np.isnan(s)
+    s = np.where(nan, 0.0, s)
+    # keys, least significant first: index, then score descending, then "is NaN"
+    return np.lexsort((np.arange(len(s)), -s, nan))
 
 
 def select_topk(score, k, tie_rel=1e-4):

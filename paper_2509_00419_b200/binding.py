@@ -127,7 +127,8 @@ def pyramid_schedule(n: int, final_ratio: float, stages: int):
 
 # ----------------------------------------------------------------------------------------------
 def score_tokens(Q, K, *, N, i0, n, q_lo, q_hi, causal=True, scale=None, lse=None,
-                 want_head=False, ws=None, dev_status=None, stream=None):
+                 want_head=False, score_out=None, head_out=None, ws=None, dev_status=None,
+                 stream=None):
     """lvlm_score_tokens.  Q [B,q_hi-q_lo,H,D] (a view with strides is fine), K [B,Hkv,cap,D].
     Returns (score [B,n], score_head [B,Hkv,n] or None)."""
     B, Nq, H, D = Q.shape
@@ -139,8 +140,11 @@ def score_tokens(Q, K, *, N, i0, n, q_lo, q_hi, causal=True, scale=None, lse=Non
     assert Q.stride(3) == 1 and K.stride(3) == 1 and K.stride(2) == D
     if scale is None:
         scale = 1.0 / math.sqrt(D)
-    score = torch.empty(B, n, dtype=torch.float32, device=Q.device)
-    head = torch.empty(B, Hkv, n, dtype=torch.float32, device=Q.device) if want_head else None
+    score = score_out if score_out is not None else \
+        torch.empty(B, n, dtype=torch.float32, device=Q.device)
+    head = head_out
+    if head is None and want_head:
+        head = torch.empty(B, Hkv, n, dtype=torch.float32, device=Q.device)
     ws, wsp, wsn = _ws(ws, OP_SCORE_TOKENS, d, Q.device)
     _check(lib().lvlm_score_tokens(_ptr(Q), _ptr(K), _ptr(lse), ctypes.byref(d),
                                    ctypes.c_float(scale), _ptr(score), _ptr(head), wsp, wsn,
@@ -148,13 +152,17 @@ def score_tokens(Q, K, *, N, i0, n, q_lo, q_hi, causal=True, scale=None, lse=Non
     return score, head
 
 
-def select_topk(score, k, *, want_kept=True, want_near=False, dev_status=None, stream=None):
+def select_topk(score, k, *, want_kept=True, want_near=False, rank_out=None, kept_out=None,
+                dev_status=None, stream=None):
     """lvlm_select_topk.  score [B,n] fp32 (row stride may exceed n).
     Returns (rank [B,n], kept_idx [B,k] or None, near_tie [B] or None)."""
     B, n = score.shape
     assert score.stride(1) == 1
-    rank = torch.empty(B, n, dtype=torch.int32, device=score.device)
-    kept = torch.empty(B, k, dtype=torch.int32, device=score.device) if want_kept else None
+    rank = rank_out if rank_out is not None else \
+        torch.empty(B, n, dtype=torch.int32, device=score.device)
+    kept = kept_out
+    if kept is None and want_kept:
+        kept = torch.empty(B, k, dtype=torch.int32, device=score.device)
     near = torch.empty(B, dtype=torch.int32, device=score.device) if want_near else None
     _check(lib().lvlm_select_topk(_ptr(score), B, n, score.stride(0), k, _ptr(rank), _ptr(kept),
                                   _ptr(near), None, 0, _ptr(dev_status), _stream(stream)),
@@ -181,8 +189,8 @@ def merged_rows(N, n, k, mode=W_LINEAR_RANK) -> int:
 
 
 def merge_compact(hidden, rank, *, i0, k, mode=W_LINEAR_RANK, Kc=None, Vc=None, pos_ids=None,
-                  w_custom=None, mass=None, in_place=False, out=None, ws=None, dev_status=None,
-                  stream=None):
+                  w_custom=None, mass=None, in_place=False, out=None, new_len=None, ws=None,
+                  dev_status=None, stream=None):
     """lvlm_merge_compact.  Returns (hidden_out or the compacted `hidden`, new_len [B]).
     With in_place=True `hidden` is compacted in place and its first new_len rows are valid.
     Kc, Vc and pos_ids are always compacted in place."""
@@ -196,7 +204,8 @@ def merge_compact(hidden, rank, *, i0, k, mode=W_LINEAR_RANK, Kc=None, Vc=None, 
         out = torch.empty(B, rows, C, dtype=hidden.dtype, device=hidden.device)
     if out is not None:
         d.out_stride_b = out.stride(0)
-    new_len = torch.empty(B, dtype=torch.int32, device=hidden.device)
+    if new_len is None:
+        new_len = torch.empty(B, dtype=torch.int32, device=hidden.device)
     ws, wsp, wsn = _ws(ws, OP_MERGE_COMPACT, d, hidden.device)
     _check(lib().lvlm_merge_compact(_ptr(hidden), _ptr(out), _ptr(Kc), _ptr(Vc), _ptr(pos_ids),
                                     _ptr(rank), ctypes.byref(d), int(mode), _ptr(w_custom),

@@ -157,6 +157,10 @@ def test_select_nonfinite_and_signed_zero():
     assert status & O.DEV_NONFINITE
     assert rank[0].tolist() == [2, 4, 3, 1, 0]      # inf, 1, +0 (idx 0), -0 (idx 2), NaN last
     assert kept[0].tolist() == [3, 4]
+    # NaN comes strictly after a genuine -inf, whatever their indices
+    s = np.array([[np.nan, -np.inf, 2.0]], np.float32)
+    rank, _, _, _ = O.select_topk(s, 1)
+    assert rank[0].tolist() == [2, 1, 0]
 
 
 def test_near_tie_counts_only_dropped_side():
