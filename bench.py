@@ -1,0 +1,534 @@
+"""Benchmark of the LightVLM hot path on B200: pyramid token reduction, one-off KV-cache
+compression and decode attention over the compressed cache, on seeded synthetic workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+                    [--extras cfg1,cfg3,cfg4,cfg5|none]
+
+Prints ONE JSON line.  A step is one pass of the whole path over one batch of the headline
+workload (cfg2: the 7B-class pyramid at layers 5/9/13, then beta-threshold compression of the
+caches of layers 6..27, then one decode step over all 28 layers).  Results for the other
+configurations (batched prefill, long decode with periodic compression, 26B-class) ride along
+under "workloads".  With N > 1 every rank runs its own replica (independent sequences, no
+collective on the data path) and rank 0 reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index=0):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+                for nm, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+class Flusher:
+    """Evicts L2 between timed iterations by overwriting a buffer larger than L2 (126 MB)."""
+    def __init__(self, device, mb=384):
+        self.buf = torch.empty(mb << 20, dtype=torch.uint8, device=device)
+        self.v = 0
+
+    def __call__(self):
+        self.v = (self.v + 1) & 0x7F
+        self.buf.fill_(self.v)
+
+
+def timed(fn, steps, warmup, flush, between=None):
+    """Mean device time (ms) of ``fn`` over ``steps`` runs after ``warmup`` runs, CUDA events on
+    the launching stream.  ``between`` (restoring tensors that are compacted in place) and the
+    L2 flush run outside the event pairs."""
+    ts = []
+    for it in range(warmup + steps):
+        if between is not None:
+            between()
+        if flush is not None:
+            flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        if it >= warmup:
+            ts.append(e0.elapsed_time(e1))
+    return float(np.mean(ts)), ts
+
+
+# ------------------------------------------------------------------------------------------
+# prefill: pyramid reduction stages
+# ------------------------------------------------------------------------------------------
+def bench_prefill(w, device, steps, warmup, flush, peaks, breakdown=True):
+    from paper_2509_00419_b200 import pipeline as P
+    run = P.PyramidPrefill(w, device)
+    g = P.capture(run.step)
+    ms, _ = timed(g.replay, steps, warmup, flush, between=run.restore)
+    res = {"ms_per_step": ms, "tokens_in": run.tokens_in,
+           "tokens_per_s": run.tokens_in / (ms * 1e-3), "launches": run.launches, "stages": []}
+    if breakdown:
+        for s, st in enumerate(run.stages):
+            hidden_in = run.hidden0 if s == 0 else run.stages[s - 1].hidden_out
+            t_sc, _ = timed(lambda: st.run_score(run.Q[s], run.K[s]), steps, warmup, flush,
+                            between=run.restore)
+            t_se, _ = timed(st.run_select, steps, warmup, flush)
+            t_me, _ = timed(lambda: st.run_merge(hidden_in, run.K[s], run.V[s], run.pos[s]),
+                            steps, warmup, flush, between=run.restore)
+            by = st.bytes_merge_hidden() + st.bytes_merge_kv()
+            res["stages"].append({
+                "n_in": st.n, "n_out": st.M, "score_ms": t_sc, "select_ms": t_se,
+                "merge_compact_ms": t_me, "merge_compact_bytes": by,
+                "merge_compact_gbs": by / (t_me * 1e6),
+                "merge_compact_frac_hbm": by / (t_me * 1e6) / peaks["hbm_gbs"],
+                "score_tflops": st.flops_score() / (t_sc * 1e9),
+                "score_frac_tensor": st.flops_score() / (t_sc * 1e9) / peaks["bf16_tflops"]})
+    return res, run
+
+
+# ------------------------------------------------------------------------------------------
+# the headline step: prefill pyramid + one-off compression + one decode step
+# ------------------------------------------------------------------------------------------
+class FullPass:
+    """Phases of one step of a workload that has reduction stages, a one-off beta compression of
+    the caches of layers kv_first_layer.. and a decode step over all layers."""
+
+    def __init__(self, w, device):
+        from paper_2509_00419_b200 import binding as L
+        from paper_2509_00419_b200 import inputs as I
+        from paper_2509_00419_b200 import pipeline as P
+        self.w, self.L, self.device = w, L, device
+        self.pre = P.PyramidPrefill(w, device)
+        # original positions of the tokens that survive each stage (one reference pass)
+        self.pre.step()
+        torch.cuda.synchronize()
+        stage_pos = [self.pre.pos[s][:, :st.Nout].clone() for s, st in enumerate(self.pre.stages)]
+        self.pre.restore()
+        stage_layers = [l for l, _ in w.stages]
+        cap = ((w.N + 64 + 63) // 64) * 64
+        self.dec = P.DecodeLayers(w.L, w.B, w.H, w.Hkv, cap, device)
+        self.lens, self.Qwin = [], []
+        pos0 = torch.arange(w.N, dtype=torch.int32, device=device)[None].repeat(w.B, 1)
+        for l in range(w.L):
+            s = sum(1 for sl in stage_layers if sl <= l)        # stages applied up to this layer
+            pos = pos0 if s == 0 else stage_pos[s - 1]
+            q, k, v = I.layer_qkv(w, l, pos, device)
+            Nl = k.shape[2]
+            self.dec.K[l, :, :, :Nl] = k
+            self.dec.V[l, :, :, :Nl] = v
+            self.dec.len[l] = Nl
+            self.Qwin.append(q[:, Nl - w.T:Nl].contiguous())
+            self.lens.append(Nl)
+        self.K0, self.V0, self.len0 = self.dec.K.clone(), self.dec.V.clone(), self.dec.len.clone()
+        first = w.kv_first_layer
+        self.first = first
+        self.e_lo = torch.full(((w.L - first) * w.B,), w.i0, dtype=torch.int32, device=device)
+        self.e_hi = torch.tensor([self.lens[l] - w.T for l in range(first, w.L) for _ in range(w.B)],
+                                 dtype=torch.int32, device=device)
+        self.ws_sc, self.sc = [], []
+        for l in range(w.L):
+            Nl = self.lens[l]
+            d = L.Dims(B=w.B, H=w.H, Hkv=w.Hkv, D=128, N=Nl, cap=cap, i0=0, n=Nl, q_lo=Nl - w.T,
+                       q_hi=Nl, causal=1)
+            self.ws_sc.append(L.alloc_workspace(L.OP_SCORE_TOKENS, d, device))
+            self.sc.append(torch.empty(w.B, Nl, dtype=torch.float32, device=device))
+        self.q_dec, self.k_new, self.v_new = [
+            torch.stack(t) for t in zip(*[tuple(x[0] for x in I.decode_inputs(w, l, 0, 1, device))
+                                          for l in range(w.L)])]
+
+    def restore(self):
+        self.pre.restore()
+        self.dec.K.copy_(self.K0); self.dec.V.copy_(self.V0); self.dec.len.copy_(self.len0)
+        self.dec.acc.zero_()
+
+    def phase_reduce(self):
+        self.pre.step()
+
+    def phase_compress(self):
+        w, L = self.w, self.L
+        for l in range(self.first, w.L):
+            Nl = self.lens[l]
+            L.score_tokens(self.Qwin[l], self.dec.K[l], N=Nl, i0=0, n=Nl, q_lo=Nl - w.T, q_hi=Nl,
+                           causal=True, score_out=self.sc[l], head_out=self.dec.acc[l][:, :, :Nl],
+                           ws=self.ws_sc[l])
+        self.dec.compress(beta=w.beta, e_lo=self.e_lo, e_hi=self.e_hi, first_layer=self.first)
+
+    def phase_decode(self):
+        self.dec.decode_step(self.q_dec, self.k_new, self.v_new, accumulate=False)
+
+    def step(self):
+        self.phase_reduce()
+        self.phase_compress()
+        self.phase_decode()
+
+    @property
+    def launches(self):
+        w = self.w
+        return self.pre.launches + 2 * (w.L - self.first) + 2 + 2 * w.L
+
+
+def bench_full(w, device, steps, warmup, flush, peaks):
+    from paper_2509_00419_b200 import pipeline as P
+    fp = FullPass(w, device)
+    g = P.capture(fp.step)
+    fp.restore()
+    ms, per_step = timed(g.replay, steps, warmup, flush, between=fp.restore)
+    # phases, timed one by one (each from the restored state it expects)
+    g_red = P.capture(fp.phase_reduce); fp.restore()
+    t_red, _ = timed(g_red.replay, steps, warmup, flush, between=fp.restore)
+    g_cmp = P.capture(fp.phase_compress); fp.restore()
+    t_cmp, _ = timed(g_cmp.replay, steps, warmup, flush, between=fp.restore)
+    fp.restore(); fp.phase_compress(); torch.cuda.synchronize()
+    lens_after = fp.dec.len.clone()
+    Kc, Vc = fp.dec.K.clone(), fp.dec.V.clone()
+
+    def restore_after_compress():
+        fp.dec.K.copy_(Kc); fp.dec.V.copy_(Vc); fp.dec.len.copy_(lens_after)
+
+    g_dec = P.capture(fp.phase_decode)
+    restore_after_compress()
+    t_dec, _ = timed(g_dec.replay, steps, warmup, flush, between=restore_after_compress)
+    kv_bytes = (int(lens_after.sum().item()) + w.L * w.B * w.Hkv) * 128 * 2 * 2
+    kept = lens_after[fp.first:].float().mean().item()
+    res = {"ms_per_step": ms, "reduce_ms": t_red, "compress_ms": t_cmp, "decode_ms": t_dec,
+           "tokens_in": fp.pre.tokens_in, "launches": fp.launches,
+           "decode_kv_bytes": kv_bytes, "decode_gbs": kv_bytes / (t_dec * 1e6),
+           "decode_frac_hbm": kv_bytes / (t_dec * 1e6) / peaks["hbm_gbs"],
+           "mean_len_after_compress": kept, "len_before": fp.lens}
+    return res, fp, per_step
+
+
+# ------------------------------------------------------------------------------------------
+# long decode with periodic compression (cfg4, and the decode half of cfg5)
+# ------------------------------------------------------------------------------------------
+def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
+    """Runs ``steps_total`` decode steps over all layers with the periodic budgeted compression;
+    every step and every compression is timed with its own event pair."""
+    from paper_2509_00419_b200 import binding as L
+    from paper_2509_00419_b200 import inputs as I
+    from paper_2509_00419_b200 import pipeline as P
+    dec = P.DecodeLayers(w.L, w.B, w.H, w.Hkv, w.cap, device)
+    pos = torch.arange(prompt_len, dtype=torch.int32, device=device)[None].repeat(w.B, 1) % w.N
+    T = min(w.T, prompt_len)
+    for l in range(w.L):
+        q, k, v = I.layer_qkv(w, l, pos, device)
+        dec.K[l, :, :, :prompt_len] = k
+        dec.V[l, :, :, :prompt_len] = v
+        sc = torch.empty(w.B, prompt_len, dtype=torch.float32, device=device)
+        L.score_tokens(q[:, prompt_len - T:].contiguous(), dec.K[l], N=prompt_len, i0=0, n=prompt_len,
+                       q_lo=prompt_len - T, q_hi=prompt_len, causal=True, score_out=sc,
+                       head_out=dec.acc[l][:, :, :prompt_len])
+    dec.len.fill_(prompt_len)
+    torch.cuda.synchronize()
+    chunk = w.trigger
+    snap = (dec.K.clone(), dec.V.clone(), dec.acc.clone())
+    qb = torch.empty(w.L, w.B, w.H, 128, dtype=torch.bfloat16, device=device)
+    kb = torch.empty(w.L, w.B, w.Hkv, 128, dtype=torch.bfloat16, device=device)
+    vb = torch.empty_like(kb)
+    g_step = P.capture(lambda: dec.decode_step(qb, kb, vb, accumulate=True))
+    g_cmp = P.capture(lambda: dec.compress(beta=1.0, budget=w.budget, recent=w.recent))
+    # the captures ran the calls once: start again from the prompt state
+    dec.K.copy_(snap[0]); dec.V.copy_(snap[1]); dec.acc.copy_(snap[2]); dec.len.fill_(prompt_len)
+    del snap
+    t_dec, t_cmp, bytes_read, n_cmp = 0.0, 0.0, 0, 0
+    cur_len = prompt_len
+    for c0 in range(0, steps_total, chunk):
+        ns = min(chunk, steps_total - c0)
+        qs, ks, vs = zip(*[I.decode_inputs(w, l, c0, ns, device) for l in range(w.L)])
+        qs, ks, vs = torch.stack(qs, 1), torch.stack(ks, 1), torch.stack(vs, 1)   # [ns, L, ...]
+        evs = []
+        if cur_len > w.budget:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g_cmp.replay(); e1.record()
+            evs.append(("c", e0, e1))
+            cur_len, n_cmp = w.budget, n_cmp + 1
+        for t in range(ns):
+            qb.copy_(qs[t]); kb.copy_(ks[t]); vb.copy_(vs[t])
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g_step.replay(); e1.record()
+            evs.append(("d", e0, e1))
+            cur_len += 1
+            bytes_read += cur_len * w.L * w.B * w.Hkv * 128 * 2 * 2
+        torch.cuda.synchronize()
+        for kind, e0, e1 in evs:
+            if kind == "d":
+                t_dec += e0.elapsed_time(e1)
+            else:
+                t_cmp += e0.elapsed_time(e1)
+    assert int(dec.len.max().item()) == cur_len and int(dec.status.item()) == 0
+    res = {"steps": steps_total, "layers": w.L, "decode_ms_total": t_dec, "compress_ms_total": t_cmp,
+           "compressions": n_cmp, "ms_per_token_step": (t_dec + t_cmp) / steps_total,
+           "decode_us_per_layer_step": t_dec * 1e3 / (steps_total * w.L),
+           "decode_kv_bytes": bytes_read, "decode_gbs": bytes_read / (t_dec * 1e6),
+           "decode_frac_hbm": bytes_read / (t_dec * 1e6) / peaks["hbm_gbs"],
+           "compress_us_per_layer": (t_cmp * 1e3 / (n_cmp * w.L)) if n_cmp else None,
+           "final_len": cur_len, "launches": steps_total * 2 * w.L + n_cmp * 2}
+    if n_cmp:
+        # bytes a compression must move per layer: read cap rows of K,V, write budget rows
+        by = w.B * w.Hkv * ((w.budget + w.trigger) + w.budget) * 128 * 2 * 2
+        res["compress_gbs"] = by * w.L * n_cmp / (t_cmp * 1e6)
+        res["compress_frac_hbm"] = res["compress_gbs"] / peaks["hbm_gbs"]
+    return res
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+def oracle_reduce_pass(w, max_stages=None):
+    """Runs the oracle's score -> select -> merge_compact chain on the workload's own tensors
+    (CPU generation), returns (seconds, image tokens reduced, description)."""
+    from oracle import lvlm_oracle as O
+    from paper_2509_00419_b200 import inputs as I
+    f64 = lambda t: t.to(torch.float64).numpy()
+    hidden = f64(I.hidden_states(w))
+    pos = np.arange(w.N, dtype=np.int32)[None].repeat(w.B, 0)
+    n, N = w.n, w.N
+    tokens, secs = 0, 0.0
+    stages = w.stages if max_stages is None else w.stages[:max_stages]
+    for layer, M in stages:
+        q, k, v = I.layer_qkv(w, layer, torch.from_numpy(pos))
+        q, k, v = f64(q[:, w.i0 + n:N]), f64(k), f64(v)
+        t0 = time.perf_counter()
+        score, _ = O.score_tokens(q, k, w.i0 + n, N, w.i0, n)
+        rank, _, _, _ = O.select_topk(score, M - 1)
+        out = O.merge_compact(hidden, rank, w.i0, n, M - 1, Kc=k, Vc=v, pos_ids=pos)
+        secs += time.perf_counter() - t0
+        tokens += w.B * n
+        hidden, pos = out["hidden"].astype(np.float64), out["pos_ids"]
+        N, n = N - (n - M), M
+    return secs, tokens, f"all {len(stages)} reduction stages of {w.name} (score, select, merge+compact of hidden, K, V), B={w.B}"
+
+
+def cpu_baseline(w):
+    secs, tokens, what = oracle_reduce_pass(w)
+    return {"value": tokens / secs, "unit": "tokens/s", "cores": torch.get_num_threads(),
+            "kind": "oracle", "sample": what, "seconds": secs}
+
+
+# ------------------------------------------------------------------------------------------
+def e2e_pass(w, device, steps, warmup):
+    """The reduction stages through the public API with HOST buffers: every step copies the
+    stage inputs from pinned host memory, runs the calls, and reads the result back."""
+    from paper_2509_00419_b200 import pipeline as P
+    run = P.PyramidPrefill(w, device)
+    host = {"hidden": run.hidden0.cpu().pin_memory(),
+            "Q": [t.cpu().pin_memory() for t in run.Q], "K": [t.cpu().pin_memory() for t in run.K0],
+            "V": [t.cpu().pin_memory() for t in run.V0], "pos": [t.cpu().pin_memory() for t in run.pos0]}
+    last = run.stages[-1]
+    out_host = torch.empty(last.hidden_out.shape, dtype=torch.bfloat16).pin_memory()
+    len_host = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    h2d = host["hidden"].numel() * 2 + sum(t.numel() * t.element_size() for k in ("Q", "K", "V", "pos")
+                                            for t in host[k])
+    d2h = out_host.numel() * 2 + len_host.numel() * 4
+
+    def step():
+        run.hidden0.copy_(host["hidden"], non_blocking=True)
+        for s in range(len(run.stages)):
+            run.Q[s].copy_(host["Q"][s], non_blocking=True)
+            run.K[s].copy_(host["K"][s], non_blocking=True)
+            run.V[s].copy_(host["V"][s], non_blocking=True)
+            run.pos[s].copy_(host["pos"][s], non_blocking=True)
+        run.step()
+        out_host.copy_(last.hidden_out, non_blocking=True)
+        len_host.copy_(last.new_len, non_blocking=True)
+
+    ms, _ = timed(step, steps, warmup, None)
+    return {"value": run.tokens_in / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "what": "reduction stages of the headline workload, inputs from pinned host memory"}
+
+
+# ------------------------------------------------------------------------------------------
+def run_reference(args, w):
+    """--impl reference: the CPU oracle, as it stands, on the same workload and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    ts, tokens, what = [], 0, ""
+    for it in range(args.warmup + args.steps):
+        secs, tokens, what = oracle_reduce_pass(w)
+        if it >= args.warmup:
+            ts.append(secs)
+    ms = float(np.mean(ts)) * 1e3
+    val = tokens / (ms * 1e-3)
+    cores = torch.get_num_threads()
+    print(json.dumps({
+        "impl": "reference", "metric": "reduced image tokens/s", "value": val, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "sample": what},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="lvlm", choices=["lvlm", "reference"])
+    ap.add_argument("--extras", default="cfg1,cfg3,cfg4,cfg5")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the decode loop length")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "lvlm" else args.warmup
+
+    from paper_2509_00419_b200 import inputs as I
+    w = I.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+        w = I.shrink(w, seed=w.seed + 1000 * rank)          # every rank its own sequences
+    from paper_2509_00419_b200 import build as Bld
+    from paper_2509_00419_b200 import binding as L
+    if rank == 0:
+        Bld.build()
+    if world > 1:
+        dist.barrier()
+    L.lib()
+    peaks = load_peaks()
+    flush = Flusher(device)
+
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    res, fp, per_step = bench_full(w, device, args.steps, args.warmup, flush, peaks)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = res["ms_per_step"]
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    tokens = res["tokens_in"] * world
+    # dominant call of the step: merge+compact of stage 1 (hidden, K, V rows), bytes per call
+    stage_break, _ = bench_prefill(w, device, args.steps, args.warmup, flush, peaks)
+    calls = []
+    for s, st in enumerate(stage_break["stages"]):
+        calls += [(f"stage{s + 1}.score", st["score_ms"]), (f"stage{s + 1}.select", st["select_ms"]),
+                  (f"stage{s + 1}.merge_compact", st["merge_compact_ms"])]
+    s1 = stage_break["stages"][0]
+    roofline = {"bound": "hbm", "kernel": "lvlm_merge_compact (stage 1: hidden out of place, K and V in place)",
+                "achieved": s1["merge_compact_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": s1["merge_compact_frac_hbm"], "traffic": None,
+                "peak_source": peaks["source"], "algorithmic_bytes": s1["merge_compact_bytes"],
+                "ms": s1["merge_compact_ms"]}
+    out = {
+        "metric": "reduced image tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "layers": w.L, "hidden": w.C, "heads": f"{w.H}/{w.Hkv}",
+                   "image_tokens": w.n, "text_tokens": w.T,
+                   "stages": [[l, m] for l, m in w.stages], "beta": w.beta,
+                   "l2": "flushed between timed iterations (384 MB overwrite)",
+                   "step": "reduce stages + score/compress layers %d..%d + one decode step over %d layers"
+                           % (w.kv_first_layer, w.L - 1, w.L)},
+        "phases_ms": {"reduce": res["reduce_ms"], "kv_compress": res["compress_ms"], "decode": res["decode_ms"]},
+        "calls_ms": dict(calls),
+        "decode": {"value": res["decode_gbs"], "unit": "GB/s", "frac_of_hbm_peak": res["decode_frac_hbm"],
+                   "kv_bytes_per_step": res["decode_kv_bytes"],
+                   "mean_len_after_compress": res["mean_len_after_compress"]},
+        "roofline": roofline, "clocks": clocks, "gpu_launches": res["launches"] * args.steps,
+        "peaks": peaks,
+    }
+    if rank == 0 and world == 1:
+        out["e2e"] = e2e_pass(w, device, args.steps, args.warmup)
+        extras = {} if args.extras in ("", "none") else {}
+        for name in [x for x in args.extras.split(",") if x and x != "none"]:
+            wx = I.WORKLOADS[name]
+            try:
+                ex = {}
+                if wx.stages:
+                    ex["prefill"], run = bench_prefill(wx, device, max(5, args.steps // 2), 3, flush, peaks)
+                    del run
+                    torch.cuda.empty_cache()
+                if wx.decode_steps > 1:
+                    prompt = wx.N if not wx.stages else wx.stages[-1][1] + wx.T + wx.i0
+                    nsteps = args.decode_steps or wx.decode_steps
+                    ex["decode_loop"] = bench_decode_loop(wx, device, flush, peaks, prompt, nsteps)
+                    torch.cuda.empty_cache()
+                extras[name] = ex
+            except Exception as e:          # an extra must not take the headline down
+                extras[name] = {"error": repr(e)}
+        out["workloads"] = extras
+        out["cpu_baseline"] = cpu_baseline(w)
+    elif rank == 0:
+        out["e2e"] = {"value": None, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                      "what": "measured at N=1 only"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

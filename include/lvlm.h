@@ -86,6 +86,7 @@ typedef struct lvlm_dims {
     int64_t kv_stride_b, kv_stride_h;            /* K,V[b][g][row][D], rows packed; default [B][Hkv][cap][D] */
     int64_t hid_stride_b;                        /* hidden[b][row][C], rows packed; default N*C */
     int64_t out_stride_b;                        /* hidden_out[b][row][C]; default (rows after the call)*C */
+    int64_t head_stride;                         /* score_head[b][g] rows; default n */
 } lvlm_dims;
 
 /* Library version string (static storage). */
@@ -113,8 +114,9 @@ size_t lvlm_workspace_bytes(int op, const lvlm_dims* d);
  *   K          [B][Hkv][cap][D] bf16, rows 0..N-1 valid (strides d->kv_stride_*)
  *   lse        optional [B][H][q_hi-q_lo] fp32: natural-log sum-exp of each row's scaled
  *              logits as produced by the attention kernel that ran before; NULL = computed here
- *   score      [B][n] fp32 out;  score_head optional [B][Hkv][n] fp32 out
- * Reads d: B,H,Hkv,D,N,cap,i0,n,q_lo,q_hi,causal,q_stride_*,kv_stride_*.
+ *   score      [B][n] fp32 out;  score_head optional [B][Hkv] rows of n fp32 out, d->head_stride apart
+ *              (a caller can point it at acc_score + i0 of a cache with head_stride = cap)
+ * Reads d: B,H,Hkv,D,N,cap,i0,n,q_lo,q_hi,causal,q_stride_*,kv_stride_*,head_stride.
  * Errors: INVALID_ARG (NULL Q/K/score, i0+n>N, q_lo>=q_hi, q_hi>N, N>cap, H%Hkv), UNSUPPORTED
  * (D!=128), ALIGNMENT, WORKSPACE.  A non-finite score sets LVLM_DEV_NONFINITE.
  */

@@ -32,7 +32,7 @@ class Dims(ctypes.Structure):
                  "recent")] + \
                [(n, ctypes.c_int64) for n in
                 ("q_stride_b", "q_stride_n", "q_stride_h", "kv_stride_b", "kv_stride_h",
-                 "hid_stride_b", "out_stride_b")]
+                 "hid_stride_b", "out_stride_b", "head_stride")]
 
 
 class LvlmError(RuntimeError):
@@ -145,6 +145,9 @@ def score_tokens(Q, K, *, N, i0, n, q_lo, q_hi, causal=True, scale=None, lse=Non
     head = head_out
     if head is None and want_head:
         head = torch.empty(B, Hkv, n, dtype=torch.float32, device=Q.device)
+    if head is not None:
+        assert head.stride(2) == 1 and head.stride(0) == Hkv * head.stride(1)
+        d.head_stride = head.stride(1)
     ws, wsp, wsn = _ws(ws, OP_SCORE_TOKENS, d, Q.device)
     _check(lib().lvlm_score_tokens(_ptr(Q), _ptr(K), _ptr(lse), ctypes.byref(d),
                                    ctypes.c_float(scale), _ptr(score), _ptr(head), wsp, wsn,

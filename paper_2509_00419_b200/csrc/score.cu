@@ -139,7 +139,7 @@ score_colsum_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
 // score[b,j] = (1/H) sum_h partial[b,h,j];  score_head[b,g,j] = sum_{h in g} partial[b,h,j].
 __global__ void score_reduce_kernel(const float* __restrict__ partial, int H, int G, int n,
                                     float* __restrict__ score, float* __restrict__ score_head,
-                                    int32_t* dev_status) {
+                                    int64_t head_stride, int32_t* dev_status) {
     const int b = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
@@ -148,7 +148,7 @@ __global__ void score_reduce_kernel(const float* __restrict__ partial, int H, in
     for (int g = 0; g < Hkv; ++g) {
         float gs = 0.f;
         for (int hh = 0; hh < G; ++hh) gs += partial[((int64_t)b * H + g * G + hh) * n + j];
-        if (score_head) score_head[((int64_t)b * Hkv + g) * n + j] = gs;
+        if (score_head) score_head[((int64_t)b * Hkv + g) * head_stride + j] = gs;
         tot += gs;
     }
     const float s = tot * (1.0f / (float)H);
@@ -174,7 +174,8 @@ lvlm_status launch_score_simt(const void* Q, const void* K, const float* lse, co
 lvlm_status launch_score_reduce(const float* partial, const lvlm_dims* d, float* score,
                                 float* score_head, int32_t* dev_status, cudaStream_t stream) {
     score_reduce_kernel<<<dim3((d->n + 255) / 256, d->B), 256, 0, stream>>>(
-        partial, d->H, d->H / d->Hkv, d->n, score, score_head, dev_status);
+        partial, d->H, d->H / d->Hkv, d->n, score, score_head,
+        d->head_stride ? d->head_stride : (int64_t)d->n, dev_status);
     return launch_status();
 }
 
@@ -194,6 +195,7 @@ extern "C" lvlm_status lvlm_score_tokens(const void* Q, const void* K, const flo
     ScoreLayout L;
     if (!Q || !K || !score || !score_layout(d, &L)) return LVLM_ERR_INVALID_ARG;
     if (d->D != kHeadDim) return LVLM_ERR_UNSUPPORTED;
+    if (d->head_stride != 0 && d->head_stride < d->n) return LVLM_ERR_INVALID_ARG;
     ScoreStrides st;
     const int Nq = d->q_hi - d->q_lo;
     st.q_sh = d->q_stride_h ? d->q_stride_h : d->D;

@@ -179,7 +179,7 @@ CFG4 = Workload("cfg4", seed=4, B=8, L=32, C=4096, H=32, Hkv=8, n=576, T=64,
                 cap=1152, beta=1.0)
 CFG5 = Workload("cfg5", seed=5, B=1, L=48, C=6144, H=48, Hkv=8, n=16384, T=256,
                 stages=((2, 4096), (12, 492)), planted=128, centroids=1024,
-                decode_steps=2048, budget=512, trigger=128, recent=128, cap=640, beta=1.0)
+                decode_steps=2048, budget=512, trigger=128, recent=128, cap=768, beta=1.0)
 
 WORKLOADS = {w.name: w for w in (CFG1, CFG2, CFG2_ALT, CFG3, CFG4, CFG5)}
 
