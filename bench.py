@@ -277,13 +277,14 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
     torch.cuda.synchronize()
     chunk = w.trigger
     snap = (dec.K.clone(), dec.V.clone(), dec.acc.clone())
-    qb = torch.empty(w.L, w.B, w.H, 128, dtype=torch.bfloat16, device=device)
-    kb = torch.empty(w.L, w.B, w.Hkv, 128, dtype=torch.bfloat16, device=device)
-    vb = torch.empty_like(kb)
+    qb = torch.zeros(w.L, w.B, w.H, 128, dtype=torch.bfloat16, device=device)
+    kb = torch.zeros(w.L, w.B, w.Hkv, 128, dtype=torch.bfloat16, device=device)
+    vb = torch.zeros_like(kb)
     g_step = P.capture(lambda: dec.decode_step(qb, kb, vb, accumulate=True))
     g_cmp = P.capture(lambda: dec.compress(beta=1.0, budget=w.budget, recent=w.recent))
     # the captures ran the calls once: start again from the prompt state
     dec.K.copy_(snap[0]); dec.V.copy_(snap[1]); dec.acc.copy_(snap[2]); dec.len.fill_(prompt_len)
+    dec.status.zero_()
     del snap
     t_dec, t_cmp, bytes_read, n_cmp = 0.0, 0.0, 0, 0
     cur_len = prompt_len
@@ -517,7 +518,8 @@ def main():
                     torch.cuda.empty_cache()
                 extras[name] = ex
             except Exception as e:          # an extra must not take the headline down
-                extras[name] = {"error": repr(e)}
+                import traceback
+                extras[name] = {"error": repr(e), "trace": traceback.format_exc()[-600:]}
         out["workloads"] = extras
         out["cpu_baseline"] = cpu_baseline(w)
     elif rank == 0:
