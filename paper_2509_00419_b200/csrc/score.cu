@@ -136,22 +136,25 @@ score_colsum_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     for (int j = tid; j < n; j += kRefRows) dst[j] = colsum[j];
 }
 
-// score[b,j] = (1/H) sum_h partial[b,h,j];  score_head[b,g,j] = sum_{h in g} partial[b,h,j].
-__global__ void score_reduce_kernel(const float* __restrict__ partial, int H, int G, int n,
-                                    float* __restrict__ score, float* __restrict__ score_head,
-                                    int64_t head_stride, int32_t* dev_status) {
+// partial holds P rows per sequence, G consecutive rows per KV group (P = H, G = group size for
+// per-head partials; P = Hkv, G = 1 for group-summed partials).
+// score[b,j] = inv_h * sum_p partial[b,p,j];  score_head[b,g,j] = sum_{p in g} partial[b,p,j].
+__global__ void score_reduce_kernel(const float* __restrict__ partial, int P, int G, int n,
+                                    float inv_h, float* __restrict__ score,
+                                    float* __restrict__ score_head, int64_t head_stride,
+                                    int32_t* dev_status) {
     const int b = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
-    const int Hkv = H / G;
+    const int Hkv = P / G;
     float tot = 0.f;
     for (int g = 0; g < Hkv; ++g) {
         float gs = 0.f;
-        for (int hh = 0; hh < G; ++hh) gs += partial[((int64_t)b * H + g * G + hh) * n + j];
+        for (int hh = 0; hh < G; ++hh) gs += partial[((int64_t)b * P + g * G + hh) * n + j];
         if (score_head) score_head[((int64_t)b * Hkv + g) * head_stride + j] = gs;
         tot += gs;
     }
-    const float s = tot * (1.0f / (float)H);
+    const float s = tot * inv_h;
     score[(int64_t)b * n + j] = s;
     if (dev_status && (__float_as_uint(s) & 0x7F800000u) == 0x7F800000u)
         atomicOr(dev_status, LVLM_DEV_NONFINITE);
@@ -171,18 +174,20 @@ lvlm_status launch_score_simt(const void* Q, const void* K, const float* lse, co
     return launch_status();
 }
 
-lvlm_status launch_score_reduce(const float* partial, const lvlm_dims* d, float* score,
-                                float* score_head, int32_t* dev_status, cudaStream_t stream) {
+lvlm_status launch_score_reduce(const float* partial, bool group_summed, const lvlm_dims* d,
+                                float* score, float* score_head, int32_t* dev_status,
+                                cudaStream_t stream) {
     score_reduce_kernel<<<dim3((d->n + 255) / 256, d->B), 256, 0, stream>>>(
-        partial, d->H, d->H / d->Hkv, d->n, score, score_head,
+        partial, group_summed ? d->Hkv : d->H, group_summed ? 1 : d->H / d->Hkv, d->n,
+        1.0f / (float)d->H, score, score_head,
         d->head_stride ? d->head_stride : (int64_t)d->n, dev_status);
     return launch_status();
 }
 
 }  // namespace lvlm
 
-// Selects the scoring kernel: 0 = automatic, 1 = CUDA-core kernel, 2 = tensor-core kernel.
-// Test hook; not part of the public header.
+// Selects the scoring kernel: 1 = CUDA-core cross-check kernel, anything else = the tensor-core
+// kernel (the product path).  Test hook; not part of the public header.
 static int g_score_impl = 0;
 extern "C" void lvlm_debug_set_score_impl(int impl) { g_score_impl = impl; }
 
@@ -209,7 +214,13 @@ extern "C" lvlm_status lvlm_score_tokens(const void* Q, const void* K, const flo
     if (!ws || !aligned256(ws) || ws_bytes < L.total) return LVLM_ERR_WORKSPACE;
     char* wsb = static_cast<char*>(ws);
     float* partial = reinterpret_cast<float*>(wsb + L.off_partial);
-    lvlm_status s = launch_score_simt(Q, K, lse, d, st, scale, partial, stream);
+    if (g_score_impl == 1) {
+        lvlm_status s = launch_score_simt(Q, K, lse, d, st, scale, partial, stream);
+        if (s != LVLM_OK) return s;
+        return launch_score_reduce(partial, false, d, score, score_head, dev_status, stream);
+    }
+    float* lse_ws = reinterpret_cast<float*>(wsb + L.off_lse);
+    lvlm_status s = launch_score_tc(Q, K, lse, d, st, scale, lse_ws, partial, dev_status, stream);
     if (s != LVLM_OK) return s;
-    return launch_score_reduce(partial, d, score, score_head, dev_status, stream);
+    return launch_score_reduce(partial, true, d, score, score_head, dev_status, stream);
 }

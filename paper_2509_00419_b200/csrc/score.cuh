@@ -9,7 +9,14 @@ struct ScoreStrides { int64_t q_sb, q_sn, q_sh, kv_sb, kv_sh; };   // elements
 
 bool score_layout(const lvlm_dims* d, ScoreLayout* L);
 
-lvlm_status launch_score_reduce(const float* partial, const lvlm_dims* d, float* score,
-                                float* score_head, int32_t* dev_status, cudaStream_t stream);
+lvlm_status launch_score_reduce(const float* partial, bool group_summed, const lvlm_dims* d,
+                                float* score, float* score_head, int32_t* dev_status,
+                                cudaStream_t stream);
+
+// Tensor-core path: pass 1 (row normalisers into lse_ws, skipped when the caller supplies lse) and
+// pass 2 (group-summed column sums into partial [B][Hkv][n]).
+lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, const lvlm_dims* d,
+                            const ScoreStrides& st, float scale, float* lse_ws, float* partial,
+                            int32_t* dev_status, cudaStream_t stream);
 
 }  // namespace lvlm

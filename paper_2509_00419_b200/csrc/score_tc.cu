@@ -1,0 +1,273 @@
+// Tensor-core scoring kernels (tcgen05 + TMEM + TMA) for lvlm_score_tokens.
+//
+// The score of an image key is a column sum of softmax probabilities (Section 3.2.1,
+// paragraph 3), so two passes over Q K^T are needed when the caller has no row normalisers:
+//   pass 1 (MODE 0)  S = Q_tile K_tile^T with QUERIES on the TMEM lanes: every epilogue thread owns
+//                    one query row and keeps its running max / sum over the key tiles -> lse.
+//   pass 2 (MODE 1)  S^T = K_tile Q_tile^T with KEYS on the TMEM lanes: every epilogue thread owns
+//                    one image key and adds exp2(logit - lse[row]) over all query rows and over
+//                    the query heads of the KV group -> group-summed column sums.
+// Both orientations are plain K-major operands (D is contiguous in Q and in K), so the same
+// pipeline serves both: the A tile is loaded once, B tiles stream through a ring of shared-memory
+// stages filled by TMA, one thread issues the MMAs into a double-buffered TMEM accumulator, and four
+// epilogue warps drain it while the next tile is being multiplied.
+#include "common.cuh"
+#include "score.cuh"
+#include "sm100.cuh"
+
+namespace lvlm {
+
+using namespace sm100;
+
+constexpr int kTile = 128;                 // rows of A, rows of B, and K (= head dim)
+constexpr int kStages = 4;                 // B-tile ring
+constexpr int kHalfBytes = kTile * 64 * 2; // one TMA box: 128 rows x 64 bf16 = 16 KB
+constexpr int kTileBytes = 2 * kHalfBytes; // 32 KB
+constexpr int kTcThreads = 192;            // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr uint32_t kTmemCols = 256;        // two 128-column fp32 accumulators
+constexpr float kLog2eT = 1.4426950408889634f;
+
+struct ScoreTcArgs {
+    int B, H, G, N, Nq, i0, n, q_lo, causal;
+    float scale_log2;
+    const float* lse_user;     // natural-log row normalisers from the caller, or NULL
+    float* lse_ws;             // [B][H][Nq] log2-domain normalisers (pass 1 writes, pass 2 reads)
+    float* partial;            // [B][Hkv][n] group-summed column sums (pass 2 writes)
+    int32_t* dev_status;
+};
+
+struct TcSmem {
+    uint64_t a_full, full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int abort;
+    float lse_s[4][2][kTile];      // per epilogue warp, per accumulator buffer
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, TcSmem* sm, int32_t* dev_status) {
+    if (sm->abort) return false;
+    if (mbar_wait(bar, parity)) return true;
+    sm->abort = 1;
+    if (dev_status) atomicOr(dev_status, LVLM_DEV_TIMEOUT);
+    return false;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kTcThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
+                const ScoreTcArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* base = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    unsigned char* sA = base;
+    unsigned char* sB = base + kTileBytes;
+    TcSmem* sm = reinterpret_cast<TcSmem*>(base + kTileBytes * (1 + kStages));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.z;
+    const int nqt = (a.Nq + kTile - 1) / kTile;
+
+    // ---- which tiles this CTA multiplies ---------------------------------------------------------
+    int nt, h = 0, g = 0, qt = 0, kt = 0, qt_min = 0, nqt_vis = 0;
+    if (MODE == 0) {
+        qt = blockIdx.x; h = blockIdx.y; g = h / a.G;
+        const int last_pos = a.q_lo + min(a.Nq, (qt + 1) * kTile) - 1;
+        const int key_end = a.causal ? min(a.N, last_pos + 1) : a.N;
+        nt = (key_end + kTile - 1) / kTile;
+    } else {
+        kt = blockIdx.x; g = blockIdx.y;
+        const int j0 = a.i0 + kt * kTile;
+        qt_min = a.causal ? max(0, (j0 - a.q_lo) / kTile) : 0;
+        nqt_vis = max(0, nqt - qt_min);
+        nt = a.G * nqt_vis;
+    }
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sm->a_full, 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sm->tmem_full[s], 1); mbar_init(&sm->tmem_empty[s], 128); }
+        sm->abort = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+        prefetch_tmap(&qmap);
+        prefetch_tmap(&kmap);
+    }
+    if (warp == 1) tmem_alloc(&sm->tmem_base, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sm->tmem_base;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0 && nt > 0) {
+            mbar_arrive_expect_tx(&sm->a_full, kTileBytes);
+            if (MODE == 0) {
+                tma_load_4d(sA, &qmap, &sm->a_full, 0, h, qt * kTile, b);
+                tma_load_4d(sA + kHalfBytes, &qmap, &sm->a_full, 64, h, qt * kTile, b);
+            } else {
+                tma_load_4d(sA, &kmap, &sm->a_full, 0, a.i0 + kt * kTile, g, b);
+                tma_load_4d(sA + kHalfBytes, &kmap, &sm->a_full, 64, a.i0 + kt * kTile, g, b);
+            }
+            for (int t = 0; t < nt; ++t) {
+                const int st = t % kStages;
+                if (t >= kStages && !wait_or_abort(&sm->empty[st], ((t / kStages) - 1) & 1, sm, a.dev_status)) break;
+                unsigned char* dst = sB + st * kTileBytes;
+                mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+                if (MODE == 0) {
+                    tma_load_4d(dst, &kmap, &sm->full[st], 0, t * kTile, g, b);
+                    tma_load_4d(dst + kHalfBytes, &kmap, &sm->full[st], 64, t * kTile, g, b);
+                } else {
+                    const int hh = g * a.G + t / nqt_vis, q2 = qt_min + t % nqt_vis;
+                    tma_load_4d(dst, &qmap, &sm->full[st], 0, hh, q2 * kTile, b);
+                    tma_load_4d(dst + kHalfBytes, &qmap, &sm->full[st], 64, hh, q2 * kTile, b);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0 && nt > 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(kTile, kTile);
+            const uint32_t a_addr = smem_u32(sA);
+            bool ok = wait_or_abort(&sm->a_full, 0, sm, a.dev_status);
+            for (int t = 0; ok && t < nt; ++t) {
+                const int st = t % kStages, buf = t & 1;
+                ok = wait_or_abort(&sm->full[st], (t / kStages) & 1, sm, a.dev_status);
+                if (ok && t >= 2) ok = wait_or_abort(&sm->tmem_empty[buf], ((t / 2) - 1) & 1, sm, a.dev_status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t b_addr = smem_u32(sB + st * kTileBytes);
+                const uint32_t d_tmem = tmem_base + buf * kTile;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
+                    mma_bf16_ss(d_tmem, smem_desc_sw128(a_addr + off), smem_desc_sw128(b_addr + off),
+                                idesc, k > 0);
+                }
+                mma_commit(&sm->empty[st]);        // the stage may be refilled once these MMAs are done
+                mma_commit(&sm->tmem_full[buf]);   // ... and the accumulator may be drained
+            }
+        }
+    } else {
+        // ================= epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 =================
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;                 // TMEM lane = row of the A tile
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        float m_run = -INFINITY, l_run = 0.f, colsum = 0.f;
+        const int my_pos = a.q_lo + qt * kTile + row;        // MODE 0: sequence position of my query
+        const int my_key = a.i0 + kt * kTile + row;          // MODE 1: my key
+        for (int t = 0; t < nt; ++t) {
+            const int buf = t & 1;
+            int q2 = 0;
+            if (MODE == 1) {
+                const int hh = g * a.G + t / nqt_vis;
+                q2 = qt_min + t % nqt_vis;
+                // every warp stages its own copy of the tile's 128 row normalisers (no block barrier)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = q2 * kTile + u * 32 + lane;
+                    float v = INFINITY;                        // rows past the window add nothing
+                    if (i < a.Nq) {
+                        const int64_t idx = ((int64_t)b * a.H + hh) * a.Nq + i;
+                        v = a.lse_user ? a.lse_user[idx] * kLog2eT : a.lse_ws[idx];
+                    }
+                    sm->lse_s[warp - 2][buf][u * 32 + lane] = v;
+                }
+                __syncwarp();
+            }
+            if (!wait_or_abort(&sm->tmem_full[buf], (t / 2) & 1, sm, a.dev_status)) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+                float v[32];
+                tmem_ld32(lane_addr + buf * kTile + c4 * 32, v);
+                tmem_ld_wait();
+                if (MODE == 0) {
+                    const int jb = t * kTile + c4 * 32;
+                    const int lim = min(a.N, a.causal ? my_pos + 1 : a.N) - jb;    // columns < lim are visible
+                    float cmax = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        v[c] = c < lim ? v[c] * a.scale_log2 : -INFINITY;
+                        cmax = fmaxf(cmax, v[c]);
+                    }
+                    const float m_new = fmaxf(m_run, cmax);
+                    if (m_new > -INFINITY) {
+                        float add = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) add += exp2f(v[c] - m_new);
+                        l_run = l_run * exp2f(m_run - m_new) + add;
+                        m_run = m_new;
+                    }
+                } else {
+                    const int ib = q2 * kTile + c4 * 32;                           // first query row of the chunk
+                    // query i sees my key iff my_key <= q_lo + i  <=>  c >= my_key - q_lo - ib
+                    const int first = a.causal ? my_key - a.q_lo - ib : 0;
+                    const float* ls = &sm->lse_s[warp - 2][buf][c4 * 32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float p = exp2f(v[c] * a.scale_log2 - ls[c]);
+                        colsum += c >= first ? p : 0.f;
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&sm->tmem_empty[buf]);
+        }
+        if (!sm->abort) {
+            if (MODE == 0) {
+                const int i = qt * kTile + row;
+                if (i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = m_run + log2f(l_run);
+            } else {
+                const int jl = kt * kTile + row;
+                if (jl < a.n) a.partial[((int64_t)b * (a.H / a.G) + g) * a.n + jl] = colsum;
+            }
+        }
+    }
+    // ---- common exit: everyone meets, then the allocating warp frees the tensor memory ----------
+    tc_fence_before();
+    __syncthreads();
+    if (sm->abort) {                              // let copies still in flight land before leaving
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, const lvlm_dims* d,
+                            const ScoreStrides& st, float scale, float* lse_ws, float* partial,
+                            int32_t* dev_status, cudaStream_t stream) {
+    const int Nq = d->q_hi - d->q_lo;
+    CUtensorMap qmap, kmap;
+    {
+        const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)d->H, (uint64_t)Nq, (uint64_t)d->B};
+        const uint64_t strides[3] = {(uint64_t)st.q_sh * 2, (uint64_t)st.q_sn * 2, (uint64_t)st.q_sb * 2};
+        const uint32_t box[4] = {64, 1, (uint32_t)kTile, 1};
+        if (!make_tmap_bf16(&qmap, Q, 4, dims, strides, box)) return LVLM_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)d->N, (uint64_t)d->Hkv, (uint64_t)d->B};
+        const uint64_t strides[3] = {(uint64_t)kHeadDim * 2, (uint64_t)st.kv_sh * 2, (uint64_t)st.kv_sb * 2};
+        const uint32_t box[4] = {64, (uint32_t)kTile, 1, 1};
+        if (!make_tmap_bf16(&kmap, K, 4, dims, strides, box)) return LVLM_ERR_CUDA;
+    }
+    ScoreTcArgs a;
+    a.B = d->B; a.H = d->H; a.G = d->H / d->Hkv; a.N = d->N; a.Nq = Nq; a.i0 = d->i0; a.n = d->n;
+    a.q_lo = d->q_lo; a.causal = d->causal; a.scale_log2 = scale * kLog2eT;
+    a.lse_user = lse; a.lse_ws = lse_ws; a.partial = partial; a.dev_status = dev_status;
+    const size_t smem = 1024 + (size_t)kTileBytes * (1 + kStages) + sizeof(TcSmem);
+    const int nqt = (Nq + kTile - 1) / kTile, nkt = (d->n + kTile - 1) / kTile;
+    if (!lse) {
+        LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<0>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        score_tc_kernel<0><<<dim3(nqt, d->H, d->B), kTcThreads, smem, stream>>>(qmap, kmap, a);
+        if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
+    }
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<1>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    score_tc_kernel<1><<<dim3(nkt, d->Hkv, d->B), kTcThreads, smem, stream>>>(qmap, kmap, a);
+    return launch_status();
+}
+
+}  // namespace lvlm
