@@ -222,12 +222,14 @@ class FullPass:
         return self.pre.launches + 2 * (w.L - self.first) + 2 + 2 * w.L
 
 
-def bench_full(w, device, steps, warmup, flush, peaks):
+def bench_full(w, device, steps, warmup, flush, peaks, phases=True):
     from paper_2509_00419_b200 import pipeline as P
     fp = FullPass(w, device)
     g = P.capture(fp.step)
     fp.restore()
     ms, per_step = timed(g.replay, steps, warmup, flush, between=fp.restore)
+    if not phases:
+        return {"ms_per_step": ms, "launches": fp.launches, "tokens_in": fp.pre.tokens_in}, fp, per_step
     # phases, timed one by one (each from the restored state it expects)
     g_red = P.capture(fp.phase_reduce); fp.restore()
     t_red, _ = timed(g_red.replay, steps, warmup, flush, between=fp.restore)
@@ -427,6 +429,11 @@ def main():
     ap.add_argument("--impl", default="lvlm", choices=["lvlm", "reference"])
     ap.add_argument("--extras", default="cfg1,cfg3,cfg4,cfg5")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode loop length")
+    ap.add_argument("--only", default="", choices=["", "step", "prefill", "decode"],
+                    help="run one piece and print its JSON: 'step' = the timed headline loop alone "
+                         "(what a profiler should see), 'prefill' = per-call times of the reduction "
+                         "stages, 'decode' = the decode loop with periodic compression")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "lvlm" else args.warmup
 
@@ -454,15 +461,32 @@ def main():
     L.lib()
     peaks = load_peaks()
     flush = Flusher(device)
+    if args.layers:
+        w = I.shrink(w, L=args.layers)
+    if args.only in ("prefill", "decode"):
+        if args.only == "prefill":
+            piece, run = bench_prefill(w, device, args.steps, args.warmup, flush, peaks)
+        else:
+            prompt = w.N if not w.stages else w.stages[-1][1] + w.T + w.i0
+            piece = bench_decode_loop(w, device, flush, peaks, prompt,
+                                      args.decode_steps or w.decode_steps)
+        print(json.dumps({"only": args.only, "workload": w.name, "layers": w.L, "result": piece,
+                          "peaks": peaks}))
+        return
 
     sampler = ClockSampler(local)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    res, fp, per_step = bench_full(w, device, args.steps, args.warmup, flush, peaks)
+    res, fp, per_step = bench_full(w, device, args.steps, args.warmup, flush, peaks,
+                                   phases=args.only != "step")
     torch.cuda.synchronize()
     clocks = sampler.stop()
+    if args.only == "step":
+        print(json.dumps({"only": "step", "workload": w.name, "ms_per_step": res["ms_per_step"],
+                          "launches_per_step": res["launches"], "clocks": clocks}))
+        return
     ms = res["ms_per_step"]
     if world > 1:
         t = torch.tensor([ms], device=device)

@@ -12,6 +12,10 @@ namespace lvlm {
 constexpr int kHeadDim = 128;
 constexpr int kMaxSortN = 16384;      // one CTA ranks at most this many 64-bit keys in shared memory
 constexpr int kMaxGroup = 8;          // query heads per KV head supported by decode attention
+// Opt-in limit of dynamic shared memory asked for every kernel that may exceed 48 KB.  The
+// attribute is a property of the function, not of a launch, so it is always set to this one
+// value: a launch recorded in a CUDA graph stays valid whatever size later calls use.
+constexpr int kMaxDynSmem = 200 * 1024;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }

@@ -140,9 +140,9 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
     if (R < 2 * a.RL) R = 2 * a.RL;
     a.R = R;
     const size_t smem = (size_t)R * V * 16;
-    if (smem > 200 * 1024) return LVLM_ERR_UNSUPPORTED;
+    if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(inplace_compact_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     dim3 grid(base1 ? 2 : 1, G, B);
     inplace_compact_kernel<<<grid, kCompactThreads, smem, stream>>>(a);
     return launch_status();

@@ -222,7 +222,7 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
     threads = threads < 64 ? 64 : (threads > 1024 ? 1024 : threads);
     const size_t smem = (size_t)P_max * 8 + (size_t)d->cap * 4;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(kv_plan_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     kv_plan_kernel<<<dim3(d->Hkv, d->B), threads, smem, stream>>>(
         acc_score, pos, len, e_lo, e_hi, d->Hkv, d->cap, d->recent, P_max, beta_ppm, budget,
         src_map, meta, nout, dev_status);

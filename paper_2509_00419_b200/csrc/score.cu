@@ -164,9 +164,9 @@ lvlm_status launch_score_simt(const void* Q, const void* K, const float* lse, co
                               const ScoreStrides& st, float scale, float* partial,
                               cudaStream_t stream) {
     const size_t smem = (size_t)((d->n + 3) & ~3) * 4 + kRefKeys * 16 * 16 + 4 * kRefKeys * 4;
-    if (smem > 200 * 1024) return LVLM_ERR_UNSUPPORTED;
+    if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_colsum_simt_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     score_colsum_simt_kernel<<<dim3(d->H, d->B), kRefRows, smem, stream>>>(
         static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K), lse, d->H,
         d->H / d->Hkv, d->N, d->i0, d->n, d->q_lo, d->q_hi, d->causal, st.q_sb, st.q_sn, st.q_sh,

@@ -81,7 +81,7 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
     threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
     const size_t smem = (size_t)P * 8 + (size_t)n * 4;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_rank_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     select_rank_kernel<<<B, threads, smem, (cudaStream_t)stream>>>(
         score, score_stride, n, k, P, rank, kept_idx, near_tie, dev_status);
     return launch_status();
