@@ -215,6 +215,38 @@ lvlm_status lvlm_decode_attn(const void* q, void* Kc, void* Vc, int32_t* len,
                              const lvlm_dims* d, float scale, void* out,
                              void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
+/*
+ * lvlm_decode_attn without a workspace argument.  The paper has no counterpart: this entry
+ * point exists for callers that cannot obtain device scratch memory at all - a plug-in inside a
+ * serving engine that owns every byte of device memory in a pool sized at start-up, a binding
+ * from a runtime that is handed raw tensor pointers but no allocator, or a decode loop that must
+ * never meet the device-wide synchronisation cudaMalloc and cudaFree imply.  It computes exactly
+ * what lvlm_decode_attn computes, with the same arguments minus `ws`/`ws_bytes`; inputs and
+ * outputs are still the caller's.
+ *
+ * The scratch is a fixed array of LVLM_STATIC_SCRATCH_BYTES inside the library image: every GPU
+ * on which the library is loaded carries it until the process exits.  A problem whose
+ * lvlm_workspace_bytes(LVLM_OP_DECODE_ATTN, d) exceeds that size is rejected with
+ * LVLM_ERR_WORKSPACE and nothing is enqueued (B * H * (cap + about 130 * splits) * 4 bytes are
+ * needed; B = 8, H = 32, cap = 1152 takes about 1.8 MiB).
+ *
+ * The first call on each device looks up the array's device address (with that device current)
+ * and remembers it; make that first call outside any stream capture.  No call allocates or frees
+ * device memory, here or in a library underneath.
+ *
+ * All calls on one device share the one array, and it keeps whatever the previous call left in
+ * it.  Nothing in it has to start at zero - every word a kernel reads was written earlier in the
+ * same call - but two calls that overlap on the GPU (different streams, no ordering between
+ * them) race on it and corrupt each other's results.  Keep calls on one stream, or order them.
+ * Errors: as lvlm_decode_attn; LVLM_ERR_WORKSPACE when the problem does not fit; LVLM_ERR_CUDA
+ * when the address lookup fails.
+ */
+#define LVLM_STATIC_SCRATCH_BYTES (4u << 20)
+lvlm_status lvlm_decode_attn_static(const void* q, void* Kc, void* Vc, int32_t* len,
+                                    const void* k_new, const void* v_new, float* acc_score,
+                                    const lvlm_dims* d, float scale, void* out,
+                                    int32_t* dev_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

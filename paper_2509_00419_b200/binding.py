@@ -22,7 +22,9 @@ W_LINEAR_RANK, W_GEOMETRIC, W_UNIFORM, W_CUSTOM, W_NEAREST_KEPT = range(5)
 OP_SCORE_TOKENS, OP_SELECT_TOPK, OP_MERGE_COMPACT, OP_KV_COMPRESS, OP_DECODE_ATTN = range(5)
 
 EXPORTS = ("lvlm_version", "lvlm_status_string", "lvlm_workspace_bytes", "lvlm_score_tokens",
-           "lvlm_select_topk", "lvlm_merge_compact", "lvlm_kv_compress", "lvlm_decode_attn")
+           "lvlm_select_topk", "lvlm_merge_compact", "lvlm_kv_compress", "lvlm_decode_attn",
+           "lvlm_decode_attn_static")
+STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class Dims(ctypes.Structure):
@@ -73,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.lvlm_kv_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, f32, i32, vp, sz, vp, vp]
         L.lvlm_decode_attn.restype = ctypes.c_int
         L.lvlm_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, f32, vp, vp, sz, vp, vp]
+        L.lvlm_decode_attn_static.restype = ctypes.c_int
+        L.lvlm_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, f32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -250,4 +254,25 @@ def decode_attn(q, Kc, Vc, length, *, k_new=None, v_new=None, acc_score=None, sc
                                   _ptr(v_new), _ptr(acc_score), ctypes.byref(d),
                                   ctypes.c_float(scale), _ptr(out), wsp, wsn, _ptr(dev_status),
                                   _stream(stream)), "lvlm_decode_attn")
+    return out
+
+
+def decode_attn_static(q, Kc, Vc, length, *, k_new=None, v_new=None, acc_score=None, scale=None,
+                       out=None, dev_status=None, stream=None):
+    """lvlm_decode_attn_static: lvlm_decode_attn for callers that have no way to get device
+    scratch memory (all of it belongs to someone else's pool, or allocating would stall the
+    device).  The scratch is a fixed array inside the library, at most STATIC_SCRATCH_BYTES per
+    problem, shared by every call on the device: calls must not overlap on the GPU.  ``out`` is
+    required to come from the caller as well when nothing may be allocated; it is created here
+    only as a convenience when omitted."""
+    B, H, D = q.shape
+    d = kv_dims(Kc, H=H)
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    if out is None:
+        out = torch.empty(B, H, D, dtype=q.dtype, device=q.device)
+    _check(lib().lvlm_decode_attn_static(_ptr(q), _ptr(Kc), _ptr(Vc), _ptr(length), _ptr(k_new),
+                                         _ptr(v_new), _ptr(acc_score), ctypes.byref(d),
+                                         ctypes.c_float(scale), _ptr(out), _ptr(dev_status),
+                                         _stream(stream)), "lvlm_decode_attn_static")
     return out

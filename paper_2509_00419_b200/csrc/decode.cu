@@ -10,6 +10,8 @@
 // barrier.  The four warps' (max, sum, output) are merged once at the end and parked per split; a
 // second kernel combines the splits in split order, writes bf16 outputs, adds the group-summed
 // probabilities to acc_score and bumps len after an append.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace lvlm {
@@ -400,4 +402,47 @@ extern "C" lvlm_status lvlm_decode_attn(const void* q, void* Kc, void* Vc, int32
     }
 #undef LVLM_DEC_CASE
     return LVLM_ERR_UNSUPPORTED;
+}
+
+// ---- decode attention for callers that cannot allocate ------------------------------------------
+// Scratch of lvlm_decode_attn_static: one array per GPU that loads the library, held until the
+// process exits.  In host code the name below is only a handle for cudaGetSymbolAddress, never a
+// pointer a kernel may be given.
+static __device__ __align__(256) unsigned char g_decode_static_scratch[LVLM_STATIC_SCRATCH_BYTES];
+
+namespace lvlm {
+
+constexpr int kMaxStaticDevices = 64;
+static void* g_static_scratch_ptr[kMaxStaticDevices];     // device address of the array, per device
+static std::mutex g_static_scratch_mutex;
+
+// Device address of the scratch array on the current device, looked up once per device.
+static lvlm_status static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxStaticDevices) return LVLM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_decode_static_scratch) != cudaSuccess || !p) return LVLM_ERR_CUDA;
+        g_static_scratch_ptr[dev] = p;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return LVLM_OK;
+}
+
+}  // namespace lvlm
+
+extern "C" lvlm_status lvlm_decode_attn_static(const void* q, void* Kc, void* Vc, int32_t* len,
+                                                const void* k_new, const void* v_new,
+                                                float* acc_score, const lvlm_dims* d, float scale,
+                                                void* out, int32_t* dev_status, void* stream) {
+    using namespace lvlm;
+    DecodeLayout L;
+    if (!decode_layout(d, &L)) return LVLM_ERR_INVALID_ARG;
+    if (L.total > (size_t)LVLM_STATIC_SCRATCH_BYTES) return LVLM_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    const lvlm_status st = static_scratch_address(&scratch);
+    if (st != LVLM_OK) return st;
+    return lvlm_decode_attn(q, Kc, Vc, len, k_new, v_new, acc_score, d, scale, out, scratch,
+                            (size_t)LVLM_STATIC_SCRATCH_BYTES, dev_status, stream);
 }
