@@ -206,7 +206,11 @@ lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, int32_t* pos,
  *            LVLM_DEV_BOUNDS is set.
  *   acc_score optional [B][Hkv][cap] fp32 in/out: entry j receives the probabilities of the
  *            group's query heads, acc_score[b,g,j] += sum_{h in g} p[b,h,j]
- * A head with len == 0 (and no append) outputs zeros.
+ * A head with len == 0 (and no append) outputs zeros.  A head whose len lies outside [0, cap]
+ * is skipped: zeros are written, nothing is appended, its len is left alone and
+ * LVLM_DEV_BOUNDS is set.
+ * Workspace: only used when acc_score is given (the scaled logits are parked there between
+ * the pass over the keys and the update of acc_score); its contents need not be zeroed.
  * Reads d: B,H,Hkv,D,cap,kv_stride_*.
  * Errors: INVALID_ARG, UNSUPPORTED (D!=128, H/Hkv > 8), ALIGNMENT, WORKSPACE.
  */
@@ -227,8 +231,8 @@ lvlm_status lvlm_decode_attn(const void* q, void* Kc, void* Vc, int32_t* len,
  * The scratch is a fixed array of LVLM_STATIC_SCRATCH_BYTES inside the library image: every GPU
  * on which the library is loaded carries it until the process exits.  A problem whose
  * lvlm_workspace_bytes(LVLM_OP_DECODE_ATTN, d) exceeds that size is rejected with
- * LVLM_ERR_WORKSPACE and nothing is enqueued (B * H * (cap + about 130 * splits) * 4 bytes are
- * needed; B = 8, H = 32, cap = 1152 takes about 1.8 MiB).
+ * LVLM_ERR_WORKSPACE and nothing is enqueued (B * H * cap * 4 bytes are needed; B = 8, H = 32,
+ * cap = 1152 takes about 1.2 MiB).
  *
  * The first call on each device looks up the array's device address (with that device current)
  * and remembers it; make that first call outside any stream capture.  No call allocates or frees

@@ -3,13 +3,16 @@
 // compression.  HBM-bound: every K and V row is read once and shared by the G query heads of
 // the group.
 //
-// Split-K: grid (splits, Hkv, B).  Inside a CTA every warp streams its own 16-key tiles through a
-// private ring of shared-memory stages (cp.async, 16-byte chunks XOR-swizzled so that ldmatrix is
-// conflict free), multiplies them with small tensor-core MMAs (the G query heads of the group are
-// the rows of a 16-row tile) and keeps an online softmax per head, so the main loop has no block
-// barrier.  The four warps' (max, sum, output) are merged once at the end and parked per split; a
-// second kernel combines the splits in split order, writes bf16 outputs, adds the group-summed
-// probabilities to acc_score and bumps len after an append.
+// One launch, split-K inside thread-block clusters.  The S CTAs of a cluster share one (sequence,
+// KV head): its ceil(len/16) key tiles are cut into S equal runs, so a ragged cache costs what
+// its own length costs.  Inside a CTA every warp streams its tiles through a private ring of
+// shared-memory stages (cp.async, 16-byte chunks XOR-swizzled so that ldmatrix is conflict free),
+// multiplies them with small tensor-core MMAs (the G query heads of the group are the rows of a
+// 16-row tile) and keeps an online softmax per head, so the main loop has no block barrier.  The
+// warps of a CTA are merged in warp order in shared memory; the CTAs of the cluster then read each
+// other's (max, sum, output) through distributed shared memory in rank order, each finishing a
+// slice of the output channels and the acc_score entries of its own keys.  Nothing goes through
+// global scratch except the scaled logits a CTA parks for its own acc_score update.
 #include <mutex>
 
 #include "common.cuh"
@@ -22,26 +25,26 @@ constexpr int kTileKeys = 16;                        // keys per warp tile
 constexpr int kStagesDec = 3;                        // stages per warp
 constexpr int kTileHalf = kTileKeys * 256;           // bytes of one K (or V) tile
 constexpr int kStageBytes = 2 * kTileHalf;           // K tile then V tile
+constexpr int kRingBytes = kDecWarps * kStagesDec * kStageBytes;
+constexpr int kDecAccFloats = 2048;                  // shared floats for merging the warps of a CTA (8 KB)
+constexpr int kDecTargetCtas = 2 * 148;              // CTAs wanted in flight: two per SM of a 148-SM part
+constexpr int kDecMaxCluster = 8;                    // portable cluster size
+constexpr int kDecMinTiles = 4;                      // a CTA's run is not made shorter than this by splitting
 constexpr float kLog2e = 1.4426950408889634f;
 
-struct DecodeLayout { int chunk, nsplit; size_t off_o, off_ml, off_s, total; };
+struct DecodeLayout { int S; size_t off_s, total; };
 
 static bool decode_layout(const lvlm_dims* d, DecodeLayout* L) {
     if (!d || d->B <= 0 || d->H <= 0 || d->Hkv <= 0 || d->H % d->Hkv || d->cap <= 0) return false;
-    // as many CTAs as fit on the GPU at once (two per SM), chunks a multiple of 64 keys so that
-    // every warp of a CTA has at least one tile
-    const int heads = d->B * d->Hkv;
-    int want = (2 * 148 + heads - 1) / heads;
-    if (want < 1) want = 1;
-    int chunk = (d->cap + want - 1) / want;
-    chunk = (chunk + 63) / 64 * 64;
-    L->chunk = chunk;
-    L->nsplit = (d->cap + chunk - 1) / chunk;
+    // cluster size: the power of two that brings the grid closest to the target without going
+    // over it, as long as a full cache still gives every CTA a few tiles
+    const int64_t heads = (int64_t)d->B * d->Hkv;
+    const int tiles = (d->cap + kTileKeys - 1) / kTileKeys;
+    int S = 1;
+    while (S < kDecMaxCluster && heads * (2 * S) <= kDecTargetCtas && tiles / (2 * S) >= kDecMinTiles) S *= 2;
+    L->S = S;
     size_t off = 0;
-    const size_t bh = (size_t)d->B * d->H;
-    L->off_o = off;  off = align_up(off + bh * L->nsplit * kHeadDim * 4, 256);
-    L->off_ml = off; off = align_up(off + bh * L->nsplit * 2 * 4, 256);
-    L->off_s = off;  off = align_up(off + bh * d->cap * 4, 256);
+    L->off_s = off; off = align_up(off + (size_t)d->B * d->H * d->cap * 4, 256);
     L->total = off;
     return true;
 }
@@ -49,6 +52,30 @@ static bool decode_layout(const lvlm_dims* d, DecodeLayout* L) {
 size_t decode_attn_workspace(const lvlm_dims* d) {
     DecodeLayout L;
     return decode_layout(d, &L) ? L.total : 0;
+}
+
+// ---- thread-block cluster primitives ---------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of every CTA of the cluster arrives and waits; shared-memory writes made before it
+// are visible to the other CTAs after it.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+// Address of my shared-memory location `saddr` in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float dsmem_ld(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
 }
 
 // 16-byte asynchronous copy; src_bytes = 0 writes zeros instead.
@@ -77,84 +104,88 @@ __device__ __forceinline__ void mma_16816(float* d, uint32_t a0, uint32_t a1, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int G>
-__global__ void __launch_bounds__(kDecThreads, 2)
-decode_split_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* Kc, __nv_bfloat16* Vc,
-                    const int32_t* __restrict__ len, const __nv_bfloat16* __restrict__ k_new,
-                    const __nv_bfloat16* __restrict__ v_new, int H, int Hkv, int cap,
-                    int64_t kv_sb, int64_t kv_sh, float scale_log2, int chunk, int nsplit,
-                    float* __restrict__ ws_o, float* __restrict__ ws_ml, float* __restrict__ ws_s,
-                    int want_logits, int32_t* dev_status) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int hd = b * Hkv + g;
-    int ln = len[hd];
-    if (ln < 0 || ln > cap) {                         // corrupt length: treat the head as empty
-        if (tid == 0 && dev_status) atomicOr(dev_status, LVLM_DEV_BOUNDS);
-        ln = 0;
-    }
-    const bool append = k_new != nullptr && ln < cap;
-    if (k_new != nullptr && ln >= cap && tid == 0 && split == 0 && dev_status)
-        atomicOr(dev_status, LVLM_DEV_BOUNDS);
-    const int ln_eff = ln + (append ? 1 : 0);
-    const int j_begin = split * chunk;
-    const int j_end = min(ln_eff, j_begin + chunk);
-    const int h0 = g * G;
+struct DecodeArgs {
+    const __nv_bfloat16* q; __nv_bfloat16* Kc; __nv_bfloat16* Vc; int32_t* len;
+    const __nv_bfloat16* k_new; const __nv_bfloat16* v_new; float* acc_score; __nv_bfloat16* out;
+    int H, Hkv, cap, S;
+    int64_t kv_sb, kv_sh;
+    float scale_log2;
+    float* ws_s;             // [B*H][cap] scaled logits (log2 domain), only with acc_score
+    int32_t* dev_status;
+};
 
-    float* my_o = ws_o + ((int64_t)(b * H + h0) * nsplit + split) * kHeadDim;      // + hh*nsplit*128
-    float* my_ml = ws_ml + ((int64_t)(b * H + h0) * nsplit + split) * 2;           // + hh*nsplit*2
-    if (j_begin >= j_end) {
-        if (tid < G) { my_ml[(int64_t)tid * nsplit * 2] = -INFINITY; my_ml[(int64_t)tid * nsplit * 2 + 1] = 0.f; }
+// grid.x = heads * S, clusters of S CTAs along x: cluster = (sequence, KV head), rank = run of tiles.
+template <int G>
+__global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const DecodeArgs a) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    float* s_acc = reinterpret_cast<float*>(smem + kRingBytes);         // [slots][G][128]; slot 0 = this CTA's output
+    float* s_wm = s_acc + kDecAccFloats;                                // [4 warps][8 heads] running max
+    float* s_wl = s_wm + kDecWarps * 8;                                 // [4 warps][8 heads] running sum
+    float* s_M = s_wl + kDecWarps * 8;                                  // [8] this CTA's max per head
+    float* s_L = s_M + 8;                                               // [8] this CTA's sum per head
+    float* s_FM = s_L + 8;                                              // [8] cluster-wide max
+    float* s_FI = s_FM + 8;                                             // [8] 1 / cluster-wide sum
+    float* s_rm = s_FI + 8;                                             // [S][8] max of every CTA of the cluster
+    float* s_rl = s_rm + 8 * kDecMaxCluster;                            // [S][8] sum of every CTA
+    float* s_rw = s_rl + 8 * kDecMaxCluster;                            // [S][8] weight of every CTA's output
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int S = a.S, H = a.H, cap = a.cap;
+    const int hd = blockIdx.x / S;
+    const int rank = (int)cluster_ctarank();
+    const int b = hd / a.Hkv, g = hd % a.Hkv, h0 = g * G;
+
+    // ---- this head's length; every CTA of the cluster takes the same decisions ---------------------------
+    int ln = a.len[hd];
+    const bool bad = ln < 0 || ln > cap;
+    if (bad) ln = 0;
+    const bool app = a.k_new != nullptr && !bad && ln < cap;
+    if (rank == 0 && tid == 0 && a.dev_status && (bad || (a.k_new != nullptr && !bad && !app)))
+        atomicOr(a.dev_status, LVLM_DEV_BOUNDS);                        // bad length, or append at capacity
+    const int lne = ln + (app ? 1 : 0);
+    if (lne == 0) {                                                     // no key at all: zeros
+        if (rank == 0)
+            for (int i = tid; i < G * kHeadDim; i += kDecThreads)
+                a.out[(int64_t)(b * H + h0) * kHeadDim + i] = __float2bfloat16_rn(0.f);
         return;
     }
-    __nv_bfloat16* Kseq = Kc + (int64_t)b * kv_sb + (int64_t)g * kv_sh;
-    __nv_bfloat16* Vseq = Vc + (int64_t)b * kv_sb + (int64_t)g * kv_sh;
-    const __nv_bfloat16* kn = append ? k_new + (int64_t)hd * kHeadDim : nullptr;
-    const __nv_bfloat16* vn = append ? v_new + (int64_t)hd * kHeadDim : nullptr;
+    const int nt = (lne + kTileKeys - 1) / kTileKeys;
+    const int per = (nt + S - 1) / S;
+    const int t_lo = min(nt, rank * per), t_hi = min(nt, t_lo + per);   // my run of tiles
 
-    // the CTA whose chunk holds row `ln` stores the appended row into the cache
-    if (append && ln >= j_begin && ln < j_end && tid < 32) {
-        const uint2 kv = reinterpret_cast<const uint2*>(kn)[lane];
-        const uint2 vv = reinterpret_cast<const uint2*>(vn)[lane];
-        reinterpret_cast<uint2*>(Kseq + (int64_t)ln * kHeadDim)[lane] = kv;
-        reinterpret_cast<uint2*>(Vseq + (int64_t)ln * kHeadDim)[lane] = vv;
-    }
+    const int64_t kv_off = (int64_t)b * a.kv_sb + (int64_t)g * a.kv_sh;
+    __nv_bfloat16* Kseq = a.Kc + kv_off;
+    __nv_bfloat16* Vseq = a.Vc + kv_off;
+    const __nv_bfloat16* kn = app ? a.k_new + (int64_t)hd * kHeadDim : nullptr;
+    const __nv_bfloat16* vn = app ? a.v_new + (int64_t)hd * kHeadDim : nullptr;
 
-    // ---- query fragments: heads of the group are rows 0..G-1 of a 16-row A tile -------------------
     const int row = lane >> 2, qd = lane & 3;
-    uint32_t qa[8][2];
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-        qa[ks][0] = qa[ks][1] = 0u;
-        if (row < G) {
-            const uint32_t* qp = reinterpret_cast<const uint32_t*>(q + (int64_t)(b * H + h0 + row) * kHeadDim);
-            qa[ks][0] = __ldg(qp + ks * 8 + qd);
-            qa[ks][1] = __ldg(qp + ks * 8 + 4 + qd);
-        }
-    }
-
-    // ---- per-warp tile ring --------------------------------------------------------------------------
     const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem) + warp * (kStagesDec * kStageBytes);
-    const int ntile_cta = (j_end - j_begin + kTileKeys - 1) / kTileKeys;
-    const int my_ntile = ntile_cta > warp ? (ntile_cta - warp + kDecWarps - 1) / kDecWarps : 0;
+    const int my_ntile = (t_hi - t_lo) > warp ? (t_hi - t_lo - warp + kDecWarps - 1) / kDecWarps : 0;
 
     auto issue = [&](int it) {                 // my it-th tile -> stage it % kStagesDec
         const uint32_t st = ring + (it % kStagesDec) * kStageBytes;
-        const int j0 = j_begin + (warp + it * kDecWarps) * kTileKeys;
+        const int j0 = (t_lo + warp + it * kDecWarps) * kTileKeys;
         // 16 rows x 16 chunks per tensor = 256 chunks, 8 per lane per tensor
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int e = u * 32 + lane;
-            const int r = e >> 4, c = e & 15;
+            const int r = e >> 4, ch = e & 15;
             const int j = j0 + r;
-            const bool ok = j < j_end;
-            const bool fresh = append && j == ln;
-            const __nv_bfloat16* ksrc = fresh ? kn : Kseq + (int64_t)(ok ? j : j_begin) * kHeadDim;
-            const __nv_bfloat16* vsrc = fresh ? vn : Vseq + (int64_t)(ok ? j : j_begin) * kHeadDim;
-            const uint32_t off = r * 256 + ((c ^ (r & 7)) << 4);
-            cp_async16_zfill(st + off, ksrc + c * 8, ok ? 16 : 0);
-            cp_async16_zfill(st + kTileHalf + off, vsrc + c * 8, ok ? 16 : 0);
+            const bool ok = j < lne;
+            const bool fresh = app && j == ln;
+            const __nv_bfloat16* ksrc = fresh ? kn : Kseq + (int64_t)(ok ? j : 0) * kHeadDim;
+            const __nv_bfloat16* vsrc = fresh ? vn : Vseq + (int64_t)(ok ? j : 0) * kHeadDim;
+            const uint32_t off = r * 256 + ((ch ^ (r & 7)) << 4);
+            cp_async16_zfill(st + off, ksrc + ch * 8, ok ? 16 : 0);
+            cp_async16_zfill(st + kTileHalf + off, vsrc + ch * 8, ok ? 16 : 0);
+        }
+        // the warp that meets the appended row also stores it into the cache
+        if (app && ln >= j0 && ln < j0 + kTileKeys) {
+            const uint2 kv = reinterpret_cast<const uint2*>(kn)[lane];
+            const uint2 vv = reinterpret_cast<const uint2*>(vn)[lane];
+            reinterpret_cast<uint2*>(Kseq + (int64_t)ln * kHeadDim)[lane] = kv;
+            reinterpret_cast<uint2*>(Vseq + (int64_t)ln * kHeadDim)[lane] = vv;
         }
     };
 #pragma unroll
@@ -163,20 +194,31 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* Kc, __nv
         cp_async_commit();
     }
 
-    float o[16][4];
+    // query fragments: heads of the group are rows 0..G-1 of a 16-row A tile
+    uint32_t qa[8][2];
 #pragma unroll
-    for (int nt = 0; nt < 16; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+    for (int ks = 0; ks < 8; ++ks) {
+        qa[ks][0] = qa[ks][1] = 0u;
+        if (row < G) {
+            const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q + (int64_t)(b * H + h0 + row) * kHeadDim);
+            qa[ks][0] = __ldg(qp + ks * 8 + qd);
+            qa[ks][1] = __ldg(qp + ks * 8 + 4 + qd);
+        }
+    }
+    float o[16][2];                            // head `row`, columns nt*8 + qd*2 + {0,1}
+#pragma unroll
+    for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = 0.f;
     float m_run = -INFINITY, l_run = 0.f;      // of head `row`; l_run is this lane's share of the sum
 
     for (int it = 0; it < my_ntile; ++it) {
         cp_async_wait<kStagesDec - 2>();
         __syncwarp();
         const uint32_t st = ring + (it % kStagesDec) * kStageBytes;
-        const int j0 = j_begin + (warp + it * kDecWarps) * kTileKeys;
-        // ---- S = Q K^T for 16 keys --------------------------------------------------------------
+        const int j0 = (t_lo + warp + it * kDecWarps) * kTileKeys;
+        // ---- S = Q K^T for 16 keys -------------------------------------------------------------------
         float s[2][4];
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+        for (int i = 0; i < 2; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
         {
             const int mi = lane >> 3, r8 = lane & 7;
             const int key = (mi >> 1) * 8 + r8;
@@ -189,19 +231,18 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* Kc, __nv
                 mma_16816(s[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
             }
         }
-        // ---- online softmax of head `row` over the tile's keys --------------------------------------
+        // ---- online softmax of head `row` over the tile's keys -------------------------------------------
         float tmax = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
+        for (int i = 0; i < 2; ++i)
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const int j = j0 + nt * 8 + qd * 2 + c;
-                float v = s[nt][c] * scale_log2;
-                if (j >= j_end) v = -INFINITY;
-                s[nt][c] = v;
+            for (int cc = 0; cc < 2; ++cc) {
+                const int j = j0 + i * 8 + qd * 2 + cc;
+                float v = s[i][cc] * a.scale_log2;
+                if (j >= lne) v = -INFINITY;
+                s[i][cc] = v;
                 tmax = fmaxf(tmax, v);
-                if (want_logits && row < G && j < j_end)
-                    ws_s[(int64_t)(b * H + h0 + row) * cap + j] = v;
+                if (a.ws_s && row < G && j < lne) a.ws_s[(int64_t)(b * H + h0 + row) * cap + j] = v;
             }
         tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 1));
         tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 2));
@@ -210,13 +251,13 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* Kc, __nv
         m_run = m_new;
         float p[2][2];
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
+        for (int i = 0; i < 2; ++i)
 #pragma unroll
-            for (int c = 0; c < 2; ++c) p[nt][c] = exp2f(s[nt][c] - m_new);
+            for (int cc = 0; cc < 2; ++cc) p[i][cc] = exp2f(s[i][cc] - m_new);
         l_run = l_run * corr + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
 #pragma unroll
-        for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
-        // ---- O += P V ---------------------------------------------------------------------------------
+        for (int i = 0; i < 16; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
+        // ---- O += P V -----------------------------------------------------------------------------------
         // P is split into a bf16 head and a bf16 remainder so that the product keeps ~16 bits
         const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]), pa2 = pack_bf16(p[1][0], p[1][1]);
         const uint32_t pr0 = pack_bf16(p[0][0] - bf16_lo(pa0), p[0][1] - bf16_hi(pa0));
@@ -229,10 +270,15 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* Kc, __nv
                 const int chunkc = 2 * dp + (mi >> 1);
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4_trans(st + kTileHalf + key * 256 + ((chunkc ^ (key & 7)) << 4), b0, b1, b2, b3);
-                mma_16816(o[2 * dp], pa0, 0u, pa2, 0u, b0, b1);
-                mma_16816(o[2 * dp + 1], pa0, 0u, pa2, 0u, b2, b3);
-                mma_16816(o[2 * dp], pr0, 0u, pr2, 0u, b0, b1);
-                mma_16816(o[2 * dp + 1], pr0, 0u, pr2, 0u, b2, b3);
+                // rows 8..15 of the MMA tile are padding: their accumulators are thrown away
+                float d0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
+                float d1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
+                mma_16816(d0, pa0, 0u, pa2, 0u, b0, b1);
+                mma_16816(d1, pa0, 0u, pa2, 0u, b2, b3);
+                mma_16816(d0, pr0, 0u, pr2, 0u, b0, b1);
+                mma_16816(d1, pr0, 0u, pr2, 0u, b2, b3);
+                o[2 * dp][0] = d0[0]; o[2 * dp][1] = d0[1];
+                o[2 * dp + 1][0] = d1[0]; o[2 * dp + 1][1] = d1[1];
             }
         }
         __syncwarp();
@@ -240,112 +286,133 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* Kc, __nv
         cp_async_commit();
     }
     cp_async_wait<0>();
-    // ---- merge the four warps, park the split's result ------------------------------------------------
+
+    // ---- merge the four warps in warp order ------------------------------------------------------------
     l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
     l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-    __syncthreads();                                       // every warp is done with its ring
-    float* wm = reinterpret_cast<float*>(smem);            // [4][8]
-    float* wl = wm + kDecWarps * 8;                        // [4][8]
-    float* wo = wl + kDecWarps * 8;                        // [4][G][128]
-    if (row < G) {
-        if (qd == 0) { wm[warp * 8 + row] = m_run; wl[warp * 8 + row] = l_run; }
-#pragma unroll
-        for (int nt = 0; nt < 16; ++nt)
-            *reinterpret_cast<float2*>(wo + ((warp * G + row) * kHeadDim) + nt * 8 + qd * 2) =
-                make_float2(o[nt][0], o[nt][1]);
-    }
+    if (row < G && qd == 0) { s_wm[warp * 8 + row] = m_run; s_wl[warp * 8 + row] = l_run; }
     __syncthreads();
-    for (int i = tid; i < G * kHeadDim; i += kDecThreads) {
-        const int hh = i / kHeadDim, dd = i % kHeadDim;
-        float M = -INFINITY;
+    {
+        // kSlots warps write side by side, the others add to them in warp order; the slots are added
+        // in slot order when they are folded into slot 0
+        constexpr int kSlots = G <= 4 ? 4 : 2;
+        float Mh = -INFINITY;
+        if (row < G) {
 #pragma unroll
-        for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, wm[w * 8 + hh]);
-        float v = 0.f, lsum = 0.f;
-#pragma unroll
-        for (int w = 0; w < kDecWarps; ++w) {
-            const float mw = wm[w * 8 + hh];
-            if (mw > -INFINITY) {
-                const float f = exp2f(mw - M);
-                v += wo[(w * G + hh) * kHeadDim + dd] * f;
-                lsum += wl[w * 8 + hh] * f;
-            }
+            for (int w = 0; w < kDecWarps; ++w) Mh = fmaxf(Mh, s_wm[w * 8 + row]);
         }
-        my_o[(int64_t)hh * nsplit * kHeadDim + dd] = v;
-        if (dd == 0) {
-            my_ml[(int64_t)hh * nsplit * 2] = M;
-            my_ml[(int64_t)hh * nsplit * 2 + 1] = lsum;
+        const float f = (row < G && m_run > -INFINITY) ? exp2f(m_run - Mh) : 0.f;
+#pragma unroll
+        for (int rnd = 0; rnd < kDecWarps / kSlots; ++rnd) {
+            if (warp / kSlots == rnd && row < G) {
+                float* slot = s_acc + (warp % kSlots) * (G * kHeadDim);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float2* dst = reinterpret_cast<float2*>(slot + row * kHeadDim + i * 8 + qd * 2);
+                    float2 v = make_float2(o[i][0] * f, o[i][1] * f);
+                    if (rnd > 0) { const float2 old = *dst; v.x += old.x; v.y += old.y; }
+                    *dst = v;
+                }
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {                  // thread = channel
+            float v = s_acc[hh * kHeadDim + tid];
+#pragma unroll
+            for (int sl = 1; sl < kSlots; ++sl) v += s_acc[sl * (G * kHeadDim) + hh * kHeadDim + tid];
+            s_acc[hh * kHeadDim + tid] = v;
+        }
+        if (tid < G) {
+            float M2 = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) M2 = fmaxf(M2, s_wm[w * 8 + tid]);
+            float Ls = 0.f;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) {
+                const float mw = s_wm[w * 8 + tid];
+                if (mw > -INFINITY) Ls += s_wl[w * 8 + tid] * exp2f(mw - M2);
+            }
+            s_M[tid] = M2;
+            s_L[tid] = Ls;
         }
     }
-}
 
-template <int G>
-__global__ void __launch_bounds__(kDecThreads)
-decode_combine_kernel(int32_t* len, int has_append, float* acc_score, int H, int Hkv, int cap,
-                      int nsplit, const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
-                      const float* __restrict__ ws_s, __nv_bfloat16* __restrict__ out) {
-    extern __shared__ float cw[];                  // [G][nsplit] weight of every split's partial output
-    __shared__ float sM[G], sInvL[G];
-    const int g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-    const int hd = b * Hkv + g;
-    int ln = len[hd];
-    if (ln < 0 || ln > cap) ln = 0;
-    const bool append = has_append && ln < cap;
-    const int ln_eff = ln + (append ? 1 : 0);
-    const int h0 = g * G;
-    const float* ml0 = ws_ml + (int64_t)(b * H + h0) * nsplit * 2;
-    // all (max, sum) pairs land in shared memory with independent loads
-    float* sml = cw + G * nsplit;                  // [G][nsplit][2]
-    for (int i = tid; i < G * nsplit * 2; i += kDecThreads) sml[i] = ml0[i];
+    // ---- combine the CTAs of the cluster in rank order through distributed shared memory ----------------
+    cluster_sync_all();
+    if (tid < 8 * S) {
+        const int r = tid >> 3, hh = tid & 7;
+        float m = -INFINITY, l = 0.f;
+        if (hh < G) {
+            m = dsmem_ld(dsmem_addr((uint32_t)__cvta_generic_to_shared(s_M + hh), r));
+            l = dsmem_ld(dsmem_addr((uint32_t)__cvta_generic_to_shared(s_L + hh), r));
+        }
+        s_rm[tid] = m;
+        s_rl[tid] = l;
+    }
     __syncthreads();
     if (tid < G) {
-        float M = -INFINITY;
-        for (int s = 0; s < nsplit; ++s) M = fmaxf(M, sml[(tid * nsplit + s) * 2]);
-        float Lsum = 0.f;
-        for (int s = 0; s < nsplit; ++s) {
-            const float l = sml[(tid * nsplit + s) * 2 + 1];
-            const float f = l > 0.f ? exp2f(sml[(tid * nsplit + s) * 2] - M) : 0.f;
-            cw[tid * nsplit + s] = f;
-            Lsum += l * f;                          // split order: fixed
+        float FM = -INFINITY;
+        for (int r = 0; r < S; ++r) FM = fmaxf(FM, s_rm[r * 8 + tid]);
+        float Ls = 0.f;
+        for (int r = 0; r < S; ++r) {
+            const float m = s_rm[r * 8 + tid];
+            const float w = m > -INFINITY ? exp2f(m - FM) : 0.f;
+            s_rw[r * 8 + tid] = w;
+            Ls += s_rl[r * 8 + tid] * w;
         }
-        const float inv = Lsum > 0.f ? 1.0f / Lsum : 0.f;
-        sM[tid] = M;
-        sInvL[tid] = inv;
+        s_FM[tid] = FM;
+        s_FI[tid] = Ls > 0.f ? 1.0f / Ls : 0.f;
     }
     __syncthreads();
+    // my slice of the output channels: element (hh, d) with hh*128 + d = rank*128 + tid (+ S*128 ...)
+    for (int idx = rank * kDecThreads + tid; idx < G * kHeadDim; idx += S * kDecThreads) {
+        const int hh = idx >> 7;
+        const uint32_t mine = (uint32_t)__cvta_generic_to_shared(s_acc + idx);
+        float x[kDecMaxCluster];
 #pragma unroll
-    for (int hh = 0; hh < G; ++hh) {
-        const float* po = ws_o + (int64_t)(b * H + h0 + hh) * nsplit * kHeadDim + tid;
+        for (int r = 0; r < kDecMaxCluster; ++r) x[r] = r < S ? dsmem_ld(dsmem_addr(mine, r)) : 0.f;
         float v = 0.f;
-        int s = 0;
-        for (; s + 3 < nsplit; s += 4) {
-            const float w0 = cw[hh * nsplit + s], w1 = cw[hh * nsplit + s + 1];
-            const float w2 = cw[hh * nsplit + s + 2], w3 = cw[hh * nsplit + s + 3];
-            const float x0 = w0 != 0.f ? po[(s + 0) * kHeadDim] : 0.f;
-            const float x1 = w1 != 0.f ? po[(s + 1) * kHeadDim] : 0.f;
-            const float x2 = w2 != 0.f ? po[(s + 2) * kHeadDim] : 0.f;
-            const float x3 = w3 != 0.f ? po[(s + 3) * kHeadDim] : 0.f;
-            v += x0 * w0; v += x1 * w1; v += x2 * w2; v += x3 * w3;
-        }
-        for (; s < nsplit; ++s) {
-            const float w0 = cw[hh * nsplit + s];
-            if (w0 != 0.f) v += po[s * kHeadDim] * w0;
-        }
-        out[(int64_t)(b * H + h0 + hh) * kHeadDim + tid] = __float2bfloat16_rn(v * sInvL[hh]);
-    }
-    if (acc_score) {
-        float* acc = acc_score + (int64_t)hd * cap;
-        for (int j = tid; j < ln_eff; j += kDecThreads) {
-            float lg[G];
 #pragma unroll
-            for (int hh = 0; hh < G; ++hh) lg[hh] = ws_s[(int64_t)(b * H + h0 + hh) * cap + j];
-            const float old = (append && j == ln) ? 0.f : acc[j];     // a new entry starts at zero
-            float p = 0.f;
+        for (int r = 0; r < kDecMaxCluster; ++r)
+            if (r < S) v += x[r] * s_rw[r * 8 + hh];
+        a.out[(int64_t)(b * H + h0) * kHeadDim + idx] = __float2bfloat16_rn(v * s_FI[hh]);
+    }
+    // the probabilities of my own keys go to acc_score
+    if (a.acc_score) {
+        float* acc = a.acc_score + (int64_t)hd * cap;
+        float il[G], mx[G];
 #pragma unroll
-            for (int hh = 0; hh < G; ++hh) p += exp2f(lg[hh] - sM[hh]) * sInvL[hh];
-            acc[j] = old + p;
+        for (int hh = 0; hh < G; ++hh) { mx[hh] = s_FM[hh]; il[hh] = s_FI[hh]; }
+        const int j_lo = t_lo * kTileKeys, j_hi = min(lne, t_hi * kTileKeys);
+        // four keys per thread per round: 4 (G + 1) independent loads in flight
+        for (int j0 = j_lo + tid; j0 < j_hi; j0 += 4 * kDecThreads) {
+            float lg[4][G], old[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = j0 + u * kDecThreads;
+                old[u] = 0.f;
+                if (j < j_hi) {
+#pragma unroll
+                    for (int hh = 0; hh < G; ++hh)
+                        lg[u][hh] = __ldcg(a.ws_s + (int64_t)(b * H + h0 + hh) * cap + j);
+                    if (!(app && j == ln)) old[u] = acc[j];                  // a new entry starts at zero
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = j0 + u * kDecThreads;
+                if (j < j_hi) {
+                    float pr = 0.f;
+#pragma unroll
+                    for (int hh = 0; hh < G; ++hh) pr += exp2f(lg[u][hh] - mx[hh]) * il[hh];
+                    acc[j] = old[u] + pr;
+                }
+            }
         }
     }
-    if (append && tid == 0) len[hd] = ln_eff;
+    if (app && rank == 0 && tid == 0) a.len[hd] = lne;    // every CTA of the cluster read it before the barrier
+    cluster_sync_all();                                   // nobody leaves while its shared memory is still read
 }
 
 template <int G>
@@ -353,24 +420,40 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
                                  const void* v_new, float* acc_score, const lvlm_dims* d, float scale,
                                  void* out, char* wsb, const DecodeLayout& L, int64_t kv_sb,
                                  int64_t kv_sh, int32_t* dev_status, cudaStream_t stream) {
-    float* ws_o = reinterpret_cast<float*>(wsb + L.off_o);
-    float* ws_ml = reinterpret_cast<float*>(wsb + L.off_ml);
-    float* ws_s = reinterpret_cast<float*>(wsb + L.off_s);
-    size_t smem = (size_t)kDecWarps * kStagesDec * kStageBytes;
-    const size_t red = (size_t)(2 * kDecWarps * 8 + kDecWarps * G * kHeadDim) * 4;
-    if (red > smem) smem = red;
-    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(decode_split_kernel<G>,
+    const size_t smem = (size_t)kRingBytes + (size_t)(kDecAccFloats + 2 * kDecWarps * 8 + 4 * 8 +
+                                                      3 * 8 * kDecMaxCluster) * 4;
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(decode_cluster_kernel<G>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_split_kernel<G><<<dim3(L.nsplit, d->Hkv, d->B), kDecThreads, smem, stream>>>(
-        static_cast<const __nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(Kc),
-        static_cast<__nv_bfloat16*>(Vc), len, static_cast<const __nv_bfloat16*>(k_new),
-        static_cast<const __nv_bfloat16*>(v_new), d->H, d->Hkv, d->cap, kv_sb, kv_sh,
-        scale * kLog2e, L.chunk, L.nsplit, ws_o, ws_ml, ws_s, acc_score != nullptr, dev_status);
-    if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
-    decode_combine_kernel<G><<<dim3(d->Hkv, d->B), kDecThreads, (size_t)G * L.nsplit * 3 * 4, stream>>>(
-        len, k_new != nullptr, acc_score, d->H, d->Hkv, d->cap, L.nsplit, ws_o, ws_ml, ws_s,
-        static_cast<__nv_bfloat16*>(out));
-    return launch_status();
+    const int64_t ctas = (int64_t)d->B * d->Hkv * L.S;
+    if (ctas > 0x7FFFFFFFll) return LVLM_ERR_UNSUPPORTED;
+    DecodeArgs a;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.Kc = static_cast<__nv_bfloat16*>(Kc);
+    a.Vc = static_cast<__nv_bfloat16*>(Vc);
+    a.len = len;
+    a.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    a.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    a.acc_score = acc_score;
+    a.out = static_cast<__nv_bfloat16*>(out);
+    a.H = d->H; a.Hkv = d->Hkv; a.cap = d->cap; a.S = L.S;
+    a.kv_sb = kv_sb; a.kv_sh = kv_sh; a.scale_log2 = scale * kLog2e;
+    a.ws_s = acc_score ? reinterpret_cast<float*>(wsb + L.off_s) : nullptr;
+    a.dev_status = dev_status;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+    cfg.blockDim = dim3(kDecThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)L.S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<G>, a));
+    return LVLM_OK;
 }
 
 }  // namespace lvlm
