@@ -66,6 +66,15 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n"
                  "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
 // Address of my shared-memory location `saddr` in the CTA of rank `rank`.
 __device__ __forceinline__ uint32_t dsmem_addr(uint32_t saddr, uint32_t rank) {
     uint32_t r;
@@ -127,7 +136,6 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
     float* s_FI = s_FM + 8;                                             // [8] 1 / cluster-wide sum
     float* s_rm = s_FI + 8;                                             // [S][8] max of every CTA of the cluster
     float* s_rl = s_rm + 8 * kDecMaxCluster;                            // [S][8] sum of every CTA
-    float* s_rw = s_rl + 8 * kDecMaxCluster;                            // [S][8] weight of every CTA's output
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.S, H = a.H, cap = a.cap;
@@ -153,6 +161,11 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
     const int per = (nt + S - 1) / S;
     const int t_lo = min(nt, rank * per), t_hi = min(nt, t_lo + per);   // my run of tiles
 
+    if (a.acc_score) {                         // my keys' acc_score entries: needed at the very end, fetched now
+        const float* acc = a.acc_score + (int64_t)hd * cap;
+        const int j_lo = t_lo * kTileKeys, j_hi = min(lne, t_hi * kTileKeys);
+        for (int j = j_lo + tid * 32; j < j_hi; j += kDecThreads * 32) prefetch_l2(acc + j);
+    }
     const int64_t kv_off = (int64_t)b * a.kv_sb + (int64_t)g * a.kv_sh;
     __nv_bfloat16* Kseq = a.Kc + kv_off;
     __nv_bfloat16* Vseq = a.Vc + kv_off;
@@ -340,7 +353,37 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
 
     // ---- combine the CTAs of the cluster in rank order through distributed shared memory ----------------
     cluster_sync_all();
-    if (tid < 8 * S) {
+    // my slice of the output channels: element (hh, d) with hh*128 + d = rank*128 + tid (+ S*128 ...).
+    // A thread fetches what it needs from every CTA in one go (max, sum and its channel) and
+    // works out the weights itself, so there is one round trip and no block barrier on this path.
+    for (int idx = rank * kDecThreads + tid; idx < G * kHeadDim; idx += S * kDecThreads) {
+        const int hh = idx >> 7;
+        const uint32_t a_o = (uint32_t)__cvta_generic_to_shared(s_acc + idx);
+        const uint32_t a_m = (uint32_t)__cvta_generic_to_shared(s_M + hh);
+        const uint32_t a_l = (uint32_t)__cvta_generic_to_shared(s_L + hh);
+        float x[kDecMaxCluster], m[kDecMaxCluster], l[kDecMaxCluster];
+#pragma unroll
+        for (int r = 0; r < kDecMaxCluster; ++r) {
+            x[r] = 0.f; m[r] = -INFINITY; l[r] = 0.f;
+            if (r < S) {
+                x[r] = dsmem_ld(dsmem_addr(a_o, r));
+                m[r] = dsmem_ld(dsmem_addr(a_m, r));
+                l[r] = dsmem_ld(dsmem_addr(a_l, r));
+            }
+        }
+        float FM = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < kDecMaxCluster; ++r) FM = fmaxf(FM, m[r]);
+        float v = 0.f, Ls = 0.f;
+#pragma unroll
+        for (int r = 0; r < kDecMaxCluster; ++r) {
+            const float w = m[r] > -INFINITY ? exp2f(m[r] - FM) : 0.f;
+            v += x[r] * w;
+            Ls += l[r] * w;
+        }
+        a.out[(int64_t)(b * H + h0) * kHeadDim + idx] = __float2bfloat16_rn(Ls > 0.f ? v / Ls : 0.f);
+    }
+    if (a.acc_score && tid < 8 * S) {          // (max, sum) of every CTA and head, for the acc_score update
         const int r = tid >> 3, hh = tid & 7;
         float m = -INFINITY, l = 0.f;
         if (hh < G) {
@@ -350,36 +393,22 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
         s_rm[tid] = m;
         s_rl[tid] = l;
     }
-    __syncthreads();
-    if (tid < G) {
-        float FM = -INFINITY;
-        for (int r = 0; r < S; ++r) FM = fmaxf(FM, s_rm[r * 8 + tid]);
-        float Ls = 0.f;
-        for (int r = 0; r < S; ++r) {
-            const float m = s_rm[r * 8 + tid];
-            const float w = m > -INFINITY ? exp2f(m - FM) : 0.f;
-            s_rw[r * 8 + tid] = w;
-            Ls += s_rl[r * 8 + tid] * w;
-        }
-        s_FM[tid] = FM;
-        s_FI[tid] = Ls > 0.f ? 1.0f / Ls : 0.f;
-    }
-    __syncthreads();
-    // my slice of the output channels: element (hh, d) with hh*128 + d = rank*128 + tid (+ S*128 ...)
-    for (int idx = rank * kDecThreads + tid; idx < G * kHeadDim; idx += S * kDecThreads) {
-        const int hh = idx >> 7;
-        const uint32_t mine = (uint32_t)__cvta_generic_to_shared(s_acc + idx);
-        float x[kDecMaxCluster];
-#pragma unroll
-        for (int r = 0; r < kDecMaxCluster; ++r) x[r] = r < S ? dsmem_ld(dsmem_addr(mine, r)) : 0.f;
-        float v = 0.f;
-#pragma unroll
-        for (int r = 0; r < kDecMaxCluster; ++r)
-            if (r < S) v += x[r] * s_rw[r * 8 + hh];
-        a.out[(int64_t)(b * H + h0) * kHeadDim + idx] = __float2bfloat16_rn(v * s_FI[hh]);
-    }
+    cluster_arrive();                          // my reads of the other CTAs' shared memory are done
     // the probabilities of my own keys go to acc_score
     if (a.acc_score) {
+        __syncthreads();
+        if (tid < G) {
+            float FM = -INFINITY;
+            for (int r = 0; r < S; ++r) FM = fmaxf(FM, s_rm[r * 8 + tid]);
+            float Ls = 0.f;
+            for (int r = 0; r < S; ++r) {
+                const float m = s_rm[r * 8 + tid];
+                if (m > -INFINITY) Ls += s_rl[r * 8 + tid] * exp2f(m - FM);
+            }
+            s_FM[tid] = FM;
+            s_FI[tid] = Ls > 0.f ? 1.0f / Ls : 0.f;
+        }
+        __syncthreads();
         float* acc = a.acc_score + (int64_t)hd * cap;
         float il[G], mx[G];
 #pragma unroll
@@ -412,7 +441,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
         }
     }
     if (app && rank == 0 && tid == 0) a.len[hd] = lne;    // every CTA of the cluster read it before the barrier
-    cluster_sync_all();                                   // nobody leaves while its shared memory is still read
+    cluster_wait();                                       // nobody leaves while its shared memory is still read
 }
 
 template <int G>
