@@ -1,19 +1,29 @@
 // In-place stable compaction of row sequences.  Every output row lies at or before its source
-// row, so one CTA can walk a sequence tile by tile in increasing order: it stages the tile's
-// source rows in shared memory, adds the merged (dropped) rows that sit in the tile's position
-// range to fp32 accumulators, and only then overwrites those positions.
+// row, so a sequence can be rewritten from the front as long as nobody overwrites a row that
+// somebody else still has to read.
+//
+// A sequence (or, for wide rows, one group of its columns: column groups never interact) is
+// walked by one thread-block cluster in super-tiles of S x R consecutive output positions, CTA
+// `rank` owning R of them.  Per super-tile every CTA stages the source rows of its positions in
+// shared memory (cp.async), adds the merged (dropped) rows that sit in its position range to fp32
+// accumulators, and only after a cluster barrier - when every CTA has its sources on chip -
+// overwrites its positions.  The sources of the next super-tile lie beyond everything written so
+// far, so they are fetched into a second buffer while the current one is being stored.
+// With many independent sequences S is 1 and the barrier is a block barrier.
 #include "compact.cuh"
 
 namespace lvlm {
 
 constexpr int kCompactThreads = 256;
-constexpr int kCompactMaxC = 4;           // 16-byte column groups per thread (rows up to 16 KB)
-constexpr int kCompactSmem = 96 * 1024;
+constexpr int kCompactMaxC = 4;              // 16-byte column groups per thread
+constexpr int kCompactBufBytes = 48 * 1024;  // one of the two staging buffers
+constexpr int kCompactMaxCluster = 8;
+constexpr int kCompactTargetCtas = 2 * 148;
 
 struct InplaceArgs {
     char* base0; char* base1;
     int64_t stride_b, stride_g;
-    int G, V, Nout, N, n, i0, merged_row, meta_stride, maps_per_g, R, CG, RL;
+    int G, V, Vsub, S, Nout, N, n, i0, merged_row, meta_stride, maps_per_g, Rmax, CG, RL;
     int64_t map_stride;
     const int32_t* src_map; const float* wgt; const int32_t* meta; const int32_t* nout;
 };
@@ -22,23 +32,57 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
     const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() {
-    asm volatile("cp.async.wait_all;\n" ::: "memory");
+__device__ __forceinline__ void cp_async_commit_group() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(const float* my_smem, uint32_t rank) {
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
 }
 
-__global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(InplaceArgs a) {
+// grid.x = column groups * S (clusters of S along x), grid.y = G (* 2 with a second tensor), grid.z = B
+__global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const InplaceArgs a) {
     extern __shared__ __align__(16) uint4 tile[];
-    const int which = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int S = a.S;
+    const int rank = (int)cluster_rank();
+    const int col = blockIdx.x / S;
+    const int which = blockIdx.y / a.G, g = blockIdx.y % a.G, b = blockIdx.z;
     char* base = (which ? a.base1 : a.base0) + (int64_t)b * a.stride_b + (int64_t)g * a.stride_g;
-    uint4* rows = reinterpret_cast<uint4*>(base);
+    const int V = a.V;
+    const int c0 = col * a.Vsub;                         // my columns: [c0, c0 + vw) of V
+    const int vw = min(a.Vsub, V - c0);
+    uint4* rows = reinterpret_cast<uint4*>(base) + c0;
     const int m = a.maps_per_g == 1 ? b : b * a.G + g;
     const int32_t* src = a.src_map + (int64_t)m * a.map_stride;
     const int Nout = a.nout ? a.nout[m] : a.Nout;
     const int o_start = a.meta[m * a.meta_stride];
     const float* w = a.wgt ? a.wgt + (int64_t)b * a.n : nullptr;
     const int Nscan = w ? a.N : Nout;
-    const int V = a.V, CG = a.CG, RL = a.RL, R = a.R;
+    const int CG = a.CG, RL = a.RL;
     const int cg = threadIdx.x % CG, rl = threadIdx.x / CG;
+
+    // rows per CTA per super-tile: everything that is left, shared out evenly, capped by the buffer
+    int R = (max(Nscan - o_start, 1) + S - 1) / S;
+    R = (R + RL - 1) / RL * RL;
+    R = min(R, a.Rmax);
+    const int Rc = R * S;
+    uint4* buf[2] = {tile, tile + (size_t)a.Rmax * a.Vsub};
+    // source row of each of my positions, three super-tiles deep: fetched two rounds ahead so
+    // that no copy ever waits for its index
+    int32_t* s_idx = reinterpret_cast<int32_t*>(tile + 2 * (size_t)a.Rmax * a.Vsub);     // [3][Rmax]
+    constexpr int kIdxPerThread = 2;                     // Rmax <= 2 * blockDim.x
 
     float acc[kCompactMaxC][8];
 #pragma unroll
@@ -46,75 +90,138 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(Inplac
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
 
-    for (int t0 = o_start; t0 < Nscan; t0 += R) {
-        for (int rr = rl; rr < R; rr += RL) {
-            const int o = t0 + rr;
-            if (o < Nout) {
-                const int s = src[o];
-                if (s >= 0 && s != o) {
+    // -1: nothing to copy (beyond the end, the merged row, or a row that stays where it is)
+    auto fetch_idx = [&](int t0, int* reg) {
 #pragma unroll
-                    for (int ci = 0; ci < kCompactMaxC; ++ci) {
-                        const int c = cg + ci * CG;
-                        if (c < V) cp_async16(&tile[rr * V + c], rows + (int64_t)s * V + c);
-                    }
+        for (int u = 0; u < kIdxPerThread; ++u) {
+            const int rr = threadIdx.x + u * kCompactThreads;
+            const int o = t0 + rank * R + rr;
+            int sidx = -1;
+            if (rr < R && o < Nout) { sidx = src[o]; if (sidx == o) sidx = -1; }
+            reg[u] = sidx;
+        }
+    };
+    auto put_idx = [&](int slot, const int* reg) {
+#pragma unroll
+        for (int u = 0; u < kIdxPerThread; ++u) {
+            const int rr = threadIdx.x + u * kCompactThreads;
+            if (rr < R) s_idx[slot * a.Rmax + rr] = reg[u];
+        }
+    };
+    auto load_tile = [&](int slot, uint4* dst) {
+        for (int rr = rl; rr < R; rr += RL) {
+            const int sidx = s_idx[slot * a.Rmax + rr];
+            if (sidx >= 0) {
+#pragma unroll
+                for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                    const int c = cg + ci * CG;
+                    if (c < vw) cp_async16(&dst[rr * a.Vsub + c], rows + (int64_t)sidx * V + c);
                 }
             }
-            if (w && o < Nscan && o >= a.i0 && o < a.i0 + a.n) {
-                const float wj = w[o - a.i0];
-                if (wj != 0.f) {
+        }
+        cp_async_commit_group();
+    };
+
+    {
+        int reg[kIdxPerThread];
+        fetch_idx(o_start, reg);
+        put_idx(0, reg);
+        fetch_idx(o_start + Rc, reg);
+        put_idx(1, reg);
+        __syncthreads();
+    }
+    load_tile(0, buf[0]);
+    int k = 0;
+    for (int t0 = o_start; t0 < Nscan; t0 += Rc, ++k) {
+        if (t0 + Rc < Nscan) load_tile((k + 1) % 3, buf[(k + 1) & 1]);
+        else cp_async_commit_group();
+        int reg[kIdxPerThread];
+        fetch_idx(t0 + 2 * Rc, reg);                  // in flight while this round runs
+        if (w) {
+            // merged rows inside my positions: read before anyone overwrites them; four rows in flight
+            for (int rb = rl; rb < R; rb += 4 * RL) {
+                float wj[4];
+                uint4 x[4][kCompactMaxC];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int rr = rb + u * RL;
+                    const int o = t0 + rank * R + rr;
+                    wj[u] = (rr < R && o < Nscan && o >= a.i0 && o < a.i0 + a.n) ? w[o - a.i0] : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int o = t0 + rank * R + rb + u * RL;
 #pragma unroll
                     for (int ci = 0; ci < kCompactMaxC; ++ci) {
                         const int c = cg + ci * CG;
-                        if (c < V) {
-                            const uint4 x = rows[(int64_t)o * V + c];
-                            acc[ci][0] = fmaf(wj, bf16_lo(x.x), acc[ci][0]); acc[ci][1] = fmaf(wj, bf16_hi(x.x), acc[ci][1]);
-                            acc[ci][2] = fmaf(wj, bf16_lo(x.y), acc[ci][2]); acc[ci][3] = fmaf(wj, bf16_hi(x.y), acc[ci][3]);
-                            acc[ci][4] = fmaf(wj, bf16_lo(x.z), acc[ci][4]); acc[ci][5] = fmaf(wj, bf16_hi(x.z), acc[ci][5]);
-                            acc[ci][6] = fmaf(wj, bf16_lo(x.w), acc[ci][6]); acc[ci][7] = fmaf(wj, bf16_hi(x.w), acc[ci][7]);
+                        x[u][ci] = (wj[u] != 0.f && c < vw) ? rows[(int64_t)o * V + c] : make_uint4(0, 0, 0, 0);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (wj[u] != 0.f) {
+#pragma unroll
+                        for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                            const uint4 xv = x[u][ci];
+                            acc[ci][0] = fmaf(wj[u], bf16_lo(xv.x), acc[ci][0]); acc[ci][1] = fmaf(wj[u], bf16_hi(xv.x), acc[ci][1]);
+                            acc[ci][2] = fmaf(wj[u], bf16_lo(xv.y), acc[ci][2]); acc[ci][3] = fmaf(wj[u], bf16_hi(xv.y), acc[ci][3]);
+                            acc[ci][4] = fmaf(wj[u], bf16_lo(xv.z), acc[ci][4]); acc[ci][5] = fmaf(wj[u], bf16_hi(xv.z), acc[ci][5]);
+                            acc[ci][6] = fmaf(wj[u], bf16_lo(xv.w), acc[ci][6]); acc[ci][7] = fmaf(wj[u], bf16_hi(xv.w), acc[ci][7]);
                         }
                     }
                 }
             }
         }
-        cp_async_wait_all();
-        __syncthreads();
+        cp_async_wait_group<1>();                     // this super-tile's sources have landed
+        cluster_barrier();                            // ... in every CTA of the cluster
+        const uint4* cur = buf[k & 1];
+        const int32_t* cur_idx = s_idx + (k % 3) * a.Rmax;
         for (int rr = rl; rr < R; rr += RL) {
-            const int o = t0 + rr;
-            if (o < Nout) {
-                const int s = src[o];
-                if (s >= 0 && s != o) {
+            if (cur_idx[rr] >= 0) {
+                const int o = t0 + rank * R + rr;
 #pragma unroll
-                    for (int ci = 0; ci < kCompactMaxC; ++ci) {
-                        const int c = cg + ci * CG;
-                        if (c < V) rows[(int64_t)o * V + c] = tile[rr * V + c];
-                    }
+                for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                    const int c = cg + ci * CG;
+                    if (c < vw) rows[(int64_t)o * V + c] = cur[rr * a.Vsub + c];
                 }
             }
         }
-        __syncthreads();
+        put_idx((k + 2) % 3, reg);
+        __syncthreads();                              // buffer and index slot are reused in the next round
     }
+    cp_async_wait_group<0>();
     if (!w) return;
-    // merged row: add the row-lane partial sums in lane order, round once, store
-    float* red = reinterpret_cast<float*>(tile);          // [RL][V*8]
+    // merged row: row lanes added in lane order, CTAs in rank order, rounded once, stored by rank 0
+    float* red = reinterpret_cast<float*>(tile);          // [RL][vw][8]
 #pragma unroll
     for (int ci = 0; ci < kCompactMaxC; ++ci) {
         const int c = cg + ci * CG;
-        if (c < V) {
+        if (c < vw) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) red[(rl * V + c) * 8 + e] = acc[ci][e];
+            for (int e = 0; e < 8; ++e) red[(rl * vw + c) * 8 + e] = acc[ci][e];
         }
     }
     __syncthreads();
-    for (int c = threadIdx.x; c < V; c += blockDim.x) {
-        float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int l = 0; l < RL; ++l)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) t[e] += red[(l * V + c) * 8 + e];
-        uint4 o;
-        o.x = pack_bf16(t[0], t[1]); o.y = pack_bf16(t[2], t[3]);
-        o.z = pack_bf16(t[4], t[5]); o.w = pack_bf16(t[6], t[7]);
-        rows[(int64_t)a.merged_row * V + c] = o;
+    float* part = red + (size_t)RL * vw * 8;              // [vw][8] this CTA's sum
+    for (int i = threadIdx.x; i < vw * 8; i += blockDim.x) {
+        float t = 0.f;
+        for (int l = 0; l < RL; ++l) t += red[l * vw * 8 + i];
+        part[i] = t;
     }
+    cluster_barrier();
+    if (rank == 0) {
+        for (int c = threadIdx.x; c < vw; c += blockDim.x) {
+            float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int r = 0; r < S; ++r)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) t[e] += ld_cluster_f32(part + c * 8 + e, r);
+            uint4 o;
+            o.x = pack_bf16(t[0], t[1]); o.y = pack_bf16(t[2], t[3]);
+            o.z = pack_bf16(t[4], t[5]); o.w = pack_bf16(t[6], t[7]);
+            rows[(int64_t)a.merged_row * V + c] = o;
+        }
+    }
+    cluster_barrier();                                    // rank 0 has read everybody's sums
 }
 
 lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, int64_t stride_g,
@@ -130,22 +237,46 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
     a.meta_stride = meta_stride; a.maps_per_g = maps_per_g;
     a.map_stride = map_stride < 0 ? N : map_stride;
     a.src_map = src_map; a.wgt = wgt; a.meta = meta; a.nout = nout;
+
+    // enough CTAs to fill the GPU: first a cluster per sequence, then column groups of wide rows
+    const int64_t nseq = (int64_t)B * G * (base1 ? 2 : 1);
+    int S = 1;
+    while (S < kCompactMaxCluster && nseq * (2 * S) <= kCompactTargetCtas && N / (2 * S) >= 32) S *= 2;
+    int Vsub = V;
+    while (Vsub > 8 && nseq * S * ((V + Vsub - 1) / Vsub) < kCompactTargetCtas / 2) Vsub = ((Vsub + 1) / 2 + 7) / 8 * 8;
+    // rows wider than the per-thread budget are always split
+    while (Vsub > kCompactMaxC * kCompactThreads) Vsub = ((Vsub + 1) / 2 + 7) / 8 * 8;
+    const int ncol = (V + Vsub - 1) / Vsub;
+    a.S = S; a.Vsub = Vsub;
     int CG = 1;
-    while (CG * 2 <= V && CG * 2 <= kCompactThreads) CG *= 2;
-    if ((V + CG - 1) / CG > kCompactMaxC) return LVLM_ERR_UNSUPPORTED;
+    while (CG * 2 <= Vsub && CG * 2 <= kCompactThreads) CG *= 2;
+    if ((Vsub + CG - 1) / CG > kCompactMaxC) return LVLM_ERR_UNSUPPORTED;
     a.CG = CG; a.RL = kCompactThreads / CG;
-    int R = kCompactSmem / (V * 16);
-    R = R > 256 ? 256 : R;
+    int R = kCompactBufBytes / (Vsub * 16);
+    R = R > 2 * kCompactThreads ? 2 * kCompactThreads : R;
     R = R / a.RL * a.RL;
-    if (R < 2 * a.RL) R = 2 * a.RL;
-    a.R = R;
-    const size_t smem = (size_t)R * V * 16;
+    if (R < a.RL) R = a.RL;
+    a.Rmax = R;
+    size_t smem = 2 * (size_t)R * Vsub * 16 + 3 * (size_t)R * 4;
+    const size_t red = ((size_t)a.RL + 1) * Vsub * 32;
+    if (red > smem) smem = red;
     if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(inplace_compact_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    dim3 grid(base1 ? 2 : 1, G, B);
-    inplace_compact_kernel<<<grid, kCompactThreads, smem, stream>>>(a);
-    return launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(ncol * S), (unsigned)(G * (base1 ? 2 : 1)), (unsigned)B);
+    cfg.blockDim = dim3(kCompactThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, inplace_compact_kernel, a));
+    return LVLM_OK;
 }
 
 }  // namespace lvlm

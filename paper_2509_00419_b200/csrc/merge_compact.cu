@@ -3,20 +3,22 @@
 // to the position ids.
 //
 // Launches: (1) a plan kernel, one CTA per sequence, turns `rank` into a source-row map for
-// every output row and a merge weight for every image token; (2) one streaming kernel moves
-// the kept rows of the hidden states and accumulates the weighted sum of the merged rows
-// (each input row is read once); (3) one kernel compacts K and V in place.
+// every output row, a destination for every input row and a merge weight for every image token;
+// (2) one streaming kernel reads every input row of the hidden states once, moves it if it is
+// kept and adds it to the weighted sum if it is merged; (3) one kernel compacts K and V in place.
 #include "common.cuh"
 #include "compact.cuh"
 
 namespace lvlm {
 
 struct MergeLayout {
-    int r1, r, Nout, V, colchunks, S;
-    size_t off_src, off_wgt, off_meta, off_partial, total;
+    int r1, r, Nout, V, cps, cl, rpc;      // CTAs per sequence, cluster size, input rows per CTA
+    size_t off_src, off_dst, off_wgt, off_meta, off_partial, total;
 };
 
-constexpr int kMergeThreads = 128;     // one 16-byte column group per thread in the merge part
+constexpr int kHidThreads = 256;       // streaming kernel: thread = 16-byte column group (+256, +512 ...)
+constexpr int kHidMaxChunks = 4;       // column groups per thread: rows up to 4 * 256 * 8 = 8192 channels
+constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
 constexpr int kMetaInts = 4;           // per sequence: first moved row, ticket counter, merged token, spare
 
 static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
@@ -27,16 +29,21 @@ static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
     L->r = L->r1 > 0 ? L->r1 - 1 : 0;
     L->Nout = d->N - L->r;
     L->V = d->C / 8;
-    L->colchunks = (L->V + kMergeThreads - 1) / kMergeThreads;
-    int S = (4 * 148 + d->B * L->colchunks - 1) / (d->B * L->colchunks);
-    const int max_by_rows = (d->n + 15) / 16;            // at least 16 image rows per slice
-    S = S > max_by_rows ? max_by_rows : S;
-    L->S = S < 1 ? 1 : (S > 128 ? 128 : S);
+    // one wave of four CTAs per SM over the whole batch, at least 8 input rows each
+    int cps = (4 * 148) / d->B;
+    const int max_by_rows = (d->N + 7) / 8;
+    cps = cps > max_by_rows ? max_by_rows : cps;
+    cps = cps < 1 ? 1 : cps;
+    L->cl = cps >= kHidCluster ? kHidCluster : 1;
+    cps = cps / L->cl * L->cl;
+    L->cps = cps;
+    L->rpc = (d->N + cps - 1) / cps;
     size_t off = 0;
     L->off_src = off;     off = align_up(off + (size_t)d->B * d->N * 4, 256);
+    L->off_dst = off;     off = align_up(off + (size_t)d->B * d->N * 4, 256);
     L->off_wgt = off;     off = align_up(off + (size_t)d->B * d->n * 4, 256);
     L->off_meta = off;    off = align_up(off + (size_t)d->B * kMetaInts * 4, 256);
-    L->off_partial = off; off = align_up(off + (size_t)d->B * L->S * d->C * 4, 256);
+    L->off_partial = off; off = align_up(off + (size_t)d->B * (cps / L->cl) * d->C * 4, 256);
     L->total = off;
     return true;
 }
@@ -78,8 +85,9 @@ __device__ __forceinline__ float merge_weight(int mode, int p, int r1, float inv
 __global__ void __launch_bounds__(1024)
 merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int i0, int n, int k,
                   int mode, float inv_sum, const float* __restrict__ w_custom,
-                  int32_t* __restrict__ src_map, float* __restrict__ wgt,
-                  int32_t* __restrict__ meta, int32_t* new_len, int32_t* dev_status) {
+                  int32_t* __restrict__ src_map, int32_t* __restrict__ dst_map,
+                  float* __restrict__ wgt, int32_t* __restrict__ meta, int32_t* new_len,
+                  int32_t* dev_status) {
     __shared__ int scan_scratch[33];
     __shared__ float fsum_scratch[33];
     __shared__ int s_first_drop, s_merged_tok, s_pos_new;
@@ -87,6 +95,7 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
     const int r1 = n - k, r = r1 - 1, Nout = N - r;
     const int32_t* rk = rank + (int64_t)b * n;
     int32_t* src = src_map + (int64_t)b * N;
+    int32_t* dst = dst_map + (int64_t)b * N;      // output row of every input row, -1 = merged away
     float* w = wgt + (int64_t)b * n;
     if (threadIdx.x == 0) { s_first_drop = n; s_merged_tok = 0; }
 
@@ -117,8 +126,10 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
         float wj = 0.f;
         if (rj < k) {
             if (off < k) src[i0 + off] = i0 + j;
+            dst[i0 + j] = off < k ? i0 + off : -1;
             ++off;
         } else {
+            dst[i0 + j] = -1;
             int p = rj - k;
             p = p < 0 ? 0 : (p >= r1 ? r1 - 1 : p);
             wj = merge_weight(mode, p, r1, inv_sum, w_custom);
@@ -126,9 +137,9 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
         w[j] = wj;
     }
     for (int o = threadIdx.x; o < Nout; o += blockDim.x) {
-        if (o < i0) src[o] = o;
+        if (o < i0) { src[o] = o; dst[o] = o; }
         else if (o == i0 + k) src[o] = -1;
-        else if (o > i0 + k) src[o] = o + r;
+        else if (o > i0 + k) { src[o] = o + r; dst[o + r] = o; }
     }
     if (bad && dev_status) atomicOr(dev_status, LVLM_DEV_BOUNDS);
     __syncthreads();
@@ -158,99 +169,152 @@ __global__ void identity_len_kernel(int32_t* new_len, int B, int N) {
     if (b < B) new_len[b] = N;
 }
 
-// Hidden states, out of place.  blockIdx.x < copy_blocks: move kept rows (one warp per output
-// row, 16-byte vectors).  The remaining blocks each own a slice of the image rows and a chunk
-// of 128 column groups, accumulate sum_j w_j x_j in fp32 in a fixed order and park the partial
-// sum; the last block to finish for a sequence adds the partials in slice order, rounds once to
-// bf16 and writes P_new.
-__global__ void __launch_bounds__(256)
-hidden_merge_compact_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
-                            int64_t hid_stride_b, int64_t out_stride_b,   // in uint4
-                            int V, int Nout, int i0, int n, int k,
-                            const int32_t* __restrict__ src_map, int N,
-                            const float* __restrict__ wgt, int32_t* meta,
-                            float* partial, int S, int colchunks, int copy_blocks,
-                            int rows_per_warp) {
-    const int b = blockIdx.y;
+__device__ __forceinline__ uint32_t hid_cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void hid_cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ float4 hid_ld_cluster_f4(const float* my_smem, uint32_t rank) {
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+    return v;
+}
+
+// Hidden states, out of place.  grid (CTAs per sequence, B), clusters of `cl` CTAs along x.  A CTA
+// owns `rpc` consecutive INPUT rows and reads each of them exactly once, four rows in flight: a kept
+// row goes to its destination, a merged row is added, times its weight, to fp32 sums the thread
+// keeps for its columns (rows in increasing order).  The CTAs of a cluster add their sums in rank
+// order through distributed shared memory and park one partial per cluster; the last cluster of
+// the sequence to finish adds the partials in cluster order, rounds once to bf16 and writes P_new.
+template <int CH>
+__global__ void __launch_bounds__(kHidThreads)
+hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
+                     int64_t hid_stride_b, int64_t out_stride_b,   // in uint4
+                     int V, int N, int i0, int n, int k, int rpc, int cl,
+                     const int32_t* __restrict__ dst_map, const float* __restrict__ wgt,
+                     int32_t* meta, float* partial) {
+    extern __shared__ __align__(16) float s_sum[];           // [V][8] this CTA's sums
+    __shared__ int s_last;
+    const int b = blockIdx.y, cta = blockIdx.x, tid = threadIdx.x;
     const uint4* hin = hidden + (int64_t)b * hid_stride_b;
     uint4* hout = out + (int64_t)b * out_stride_b;
-    if ((int)blockIdx.x < copy_blocks) {
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        const int nwarp = blockDim.x >> 5;
-        const int32_t* src = src_map + (int64_t)b * N;
-        int o = ((int)blockIdx.x * nwarp + warp) * rows_per_warp;
-        const int o_end = min(Nout, o + rows_per_warp);
-        for (; o < o_end; ++o) {
-            const int s = src[o];
-            if (s < 0) continue;
-            const uint4* srow = hin + (int64_t)s * V;
-            uint4* drow = hout + (int64_t)o * V;
-            int v = lane;
-            for (; v + 96 < V; v += 128) {
-                const uint4 a0 = __ldg(srow + v), a1 = __ldg(srow + v + 32);
-                const uint4 a2 = __ldg(srow + v + 64), a3 = __ldg(srow + v + 96);
-                drow[v] = a0; drow[v + 32] = a1; drow[v + 64] = a2; drow[v + 96] = a3;
-            }
-            for (; v < V; v += 32) drow[v] = __ldg(srow + v);
-        }
-        return;
-    }
-    // ---- merge part -------------------------------------------------------------------
-    if (threadIdx.x >= kMergeThreads) return;
-    const int mb = (int)blockIdx.x - copy_blocks;
-    const int slice = mb / colchunks, chunk = mb % colchunks;
-    const int cg = chunk * kMergeThreads + threadIdx.x;
-    const int rows_per_slice = (n + S - 1) / S;
-    const int j0 = min(n, slice * rows_per_slice), j1 = min(n, j0 + rows_per_slice);
-    const float* w = wgt + (int64_t)b * n;
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (cg < V) {
-        const uint4* col = hin + (int64_t)i0 * V + cg;
-        int j = j0;
-        for (; j + 3 < j1; j += 4) {
-            float wj[4];
-            uint4 x[4];
+    const int32_t* dst = dst_map + (int64_t)b * N;
+    const float* w = wgt + (int64_t)b * n - i0;               // indexed by sequence position
+    const int i_lo = min(N, cta * rpc), i_hi = min(N, i_lo + rpc);
+
+    float acc[CH][8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                wj[u] = w[j + u];
-                x[u] = wj[u] != 0.f ? __ldg(col + (int64_t)(j + u) * V) : make_uint4(0, 0, 0, 0);
-            }
+    for (int ci = 0; ci < CH; ++ci)
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                acc[0] = fmaf(wj[u], bf16_lo(x[u].x), acc[0]); acc[1] = fmaf(wj[u], bf16_hi(x[u].x), acc[1]);
-                acc[2] = fmaf(wj[u], bf16_lo(x[u].y), acc[2]); acc[3] = fmaf(wj[u], bf16_hi(x[u].y), acc[3]);
-                acc[4] = fmaf(wj[u], bf16_lo(x[u].z), acc[4]); acc[5] = fmaf(wj[u], bf16_hi(x[u].z), acc[5]);
-                acc[6] = fmaf(wj[u], bf16_lo(x[u].w), acc[6]); acc[7] = fmaf(wj[u], bf16_hi(x[u].w), acc[7]);
+        for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
+
+    for (int ib = i_lo; ib < i_hi; ib += 4) {
+        int d[4];
+        float wj[4];
+        uint4 x[4][CH];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = ib + u;
+            d[u] = i < i_hi ? dst[i] : -2;
+            wj[u] = (i < i_hi && i >= i0 && i < i0 + n) ? w[i] : 0.f;
+#pragma unroll
+            for (int ci = 0; ci < CH; ++ci) {
+                const int c = tid + ci * kHidThreads;
+                x[u][ci] = (i < i_hi && c < V) ? __ldg(hin + (int64_t)i * V + c) : make_uint4(0, 0, 0, 0);
             }
         }
-        for (; j < j1; ++j) {
-            const float wj = w[j];
-            if (wj == 0.f) continue;
-            const uint4 x = __ldg(col + (int64_t)j * V);
-            acc[0] = fmaf(wj, bf16_lo(x.x), acc[0]); acc[1] = fmaf(wj, bf16_hi(x.x), acc[1]);
-            acc[2] = fmaf(wj, bf16_lo(x.y), acc[2]); acc[3] = fmaf(wj, bf16_hi(x.y), acc[3]);
-            acc[4] = fmaf(wj, bf16_lo(x.z), acc[4]); acc[5] = fmaf(wj, bf16_hi(x.z), acc[5]);
-            acc[6] = fmaf(wj, bf16_lo(x.w), acc[6]); acc[7] = fmaf(wj, bf16_hi(x.w), acc[7]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (d[u] >= 0) {
+#pragma unroll
+                for (int ci = 0; ci < CH; ++ci) {
+                    const int c = tid + ci * kHidThreads;
+                    if (c < V) hout[(int64_t)d[u] * V + c] = x[u][ci];
+                }
+            } else if (d[u] == -1) {
+#pragma unroll
+                for (int ci = 0; ci < CH; ++ci) {
+                    acc[ci][0] = fmaf(wj[u], bf16_lo(x[u][ci].x), acc[ci][0]); acc[ci][1] = fmaf(wj[u], bf16_hi(x[u][ci].x), acc[ci][1]);
+                    acc[ci][2] = fmaf(wj[u], bf16_lo(x[u][ci].y), acc[ci][2]); acc[ci][3] = fmaf(wj[u], bf16_hi(x[u][ci].y), acc[ci][3]);
+                    acc[ci][4] = fmaf(wj[u], bf16_lo(x[u][ci].z), acc[ci][4]); acc[ci][5] = fmaf(wj[u], bf16_hi(x[u][ci].z), acc[ci][5]);
+                    acc[ci][6] = fmaf(wj[u], bf16_lo(x[u][ci].w), acc[ci][6]); acc[ci][7] = fmaf(wj[u], bf16_hi(x[u][ci].w), acc[ci][7]);
+                }
+            }
         }
-        float4* dst = reinterpret_cast<float4*>(partial + ((int64_t)(b * S + slice) * V + cg) * 8);
-        dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
     }
-    // ---- last block of this sequence finalises P_new ------------------------------------
-    __shared__ int s_last;
+
+    // ---- clusters that touch the image span contribute a partial sum ---------------------------------
+    const int rows_per_cluster = rpc * cl;
+    const int cluster = cta / cl;
+    const int q_first = i0 / rows_per_cluster, q_last = (i0 + n - 1) / rows_per_cluster;
+    if (cluster < q_first || cluster > q_last) return;        // the whole cluster leaves together
+    const int rank = (int)hid_cluster_rank();
+#pragma unroll
+    for (int ci = 0; ci < CH; ++ci) {
+        const int c = tid + ci * kHidThreads;
+        if (c < V) {
+            *reinterpret_cast<float4*>(s_sum + c * 8) = make_float4(acc[ci][0], acc[ci][1], acc[ci][2], acc[ci][3]);
+            *reinterpret_cast<float4*>(s_sum + c * 8 + 4) = make_float4(acc[ci][4], acc[ci][5], acc[ci][6], acc[ci][7]);
+        }
+    }
+    hid_cluster_barrier();
+    if (rank == 0) {
+        float* my_partial = partial + ((int64_t)b * gridDim.x / cl + cluster) * V * 8;
+#pragma unroll
+        for (int ci = 0; ci < CH; ++ci) {
+            const int c = tid + ci * kHidThreads;
+            if (c < V) {
+                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+                for (int r = 0; r < cl; ++r) {
+                    const float4 a0 = hid_ld_cluster_f4(s_sum + c * 8, r), a1 = hid_ld_cluster_f4(s_sum + c * 8 + 4, r);
+                    lo.x += a0.x; lo.y += a0.y; lo.z += a0.z; lo.w += a0.w;
+                    hi.x += a1.x; hi.y += a1.y; hi.z += a1.z; hi.w += a1.w;
+                }
+                *reinterpret_cast<float4*>(my_partial + c * 8) = lo;
+                *reinterpret_cast<float4*>(my_partial + c * 8 + 4) = hi;
+            }
+        }
+    }
+    hid_cluster_barrier();                                    // rank 0 has read every CTA's sums
+    if (rank != 0) return;
+    // ---- the last cluster of this sequence finalises P_new ------------------------------------------------
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         const int ticket = atomicAdd(&meta[b * kMetaInts + 1], 1);
-        s_last = ticket == S * colchunks - 1;
+        s_last = ticket == q_last - q_first;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    for (int c = threadIdx.x; c < V; c += kMergeThreads) {
+#pragma unroll 1
+    for (int ci = 0; ci < CH; ++ci) {
+        const int c = tid + ci * kHidThreads;
+        if (c >= V) break;
         float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int s = 0; s < S; ++s) {
-            const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)(b * S + s) * V + c) * 8);
+        int q = q_first;
+        for (; q + 3 <= q_last; q += 4) {                     // four partials in flight
+            float4 lo[4], hi[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)b * gridDim.x / cl + q + u) * V * 8 + c * 8);
+                lo[u] = __ldcg(p); hi[u] = __ldcg(p + 1);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                t[0] += lo[u].x; t[1] += lo[u].y; t[2] += lo[u].z; t[3] += lo[u].w;
+                t[4] += hi[u].x; t[5] += hi[u].y; t[6] += hi[u].z; t[7] += hi[u].w;
+            }
+        }
+        for (; q <= q_last; ++q) {
+            const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)b * gridDim.x / cl + q) * V * 8 + c * 8);
             const float4 lo = __ldcg(p), hi = __ldcg(p + 1);
             t[0] += lo.x; t[1] += lo.y; t[2] += lo.z; t[3] += lo.w;
             t[4] += hi.x; t[5] += hi.y; t[6] += hi.z; t[7] += hi.w;
@@ -260,7 +324,32 @@ hidden_merge_compact_kernel(const uint4* __restrict__ hidden, uint4* __restrict_
         o.z = pack_bf16(t[4], t[5]); o.w = pack_bf16(t[6], t[7]);
         hout[(int64_t)(i0 + k) * V + c] = o;
     }
-    if (threadIdx.x == 0) meta[b * kMetaInts + 1] = 0;
+    if (tid == 0) meta[b * kMetaInts + 1] = 0;
+}
+
+template <int CH>
+static lvlm_status launch_hidden_stream(const void* hidden, void* hidden_out, int64_t hid_sb, int64_t out_sb,
+                                        const lvlm_dims* d, const MergeLayout& L, const int32_t* dst_map,
+                                        const float* wgt, int32_t* meta, float* partial, cudaStream_t stream) {
+    const size_t smem = (size_t)L.V * 32;
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(hidden_stream_kernel<CH>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)L.cps, (unsigned)d->B, 1);
+    cfg.blockDim = dim3(kHidThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)L.cl;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, hidden_stream_kernel<CH>, static_cast<const uint4*>(hidden),
+                                           static_cast<uint4*>(hidden_out), hid_sb / 8, out_sb / 8, L.V, d->N,
+                                           d->i0, d->n, d->k, L.rpc, L.cl, dst_map, wgt, meta, partial));
+    return LVLM_OK;
 }
 
 }  // namespace lvlm
@@ -305,6 +394,7 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     if (!ws || !aligned256(ws) || ws_bytes < L.total) return LVLM_ERR_WORKSPACE;
     char* wsb = static_cast<char*>(ws);
     int32_t* src_map = reinterpret_cast<int32_t*>(wsb + L.off_src);
+    int32_t* dst_map = reinterpret_cast<int32_t*>(wsb + L.off_dst);
     float* wgt = reinterpret_cast<float*>(wsb + L.off_wgt);
     int32_t* meta = reinterpret_cast<int32_t*>(wsb + L.off_meta);
     float* partial = reinterpret_cast<float*>(wsb + L.off_partial);
@@ -314,22 +404,22 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     else if (mode == LVLM_W_UNIFORM) inv_sum = (float)(1.0 / (double)L.r1);
     const int plan_threads = d->n >= 1024 ? 1024 : (d->n <= 128 ? 128 : ((d->n + 31) / 32) * 32);
     merge_plan_kernel<<<d->B, plan_threads, 0, stream>>>(rank, pos_ids, d->N, d->i0, d->n, d->k,
-                                                         (int)mode, inv_sum, w_custom, src_map, wgt,
-                                                         meta, new_len, dev_status);
+                                                         (int)mode, inv_sum, w_custom, src_map, dst_map,
+                                                         wgt, meta, new_len, dev_status);
     if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
 
     if (hidden_out) {
-        // rows per warp chosen so that the grid has a few CTAs per SM when the job allows
-        const int warps = 8;
-        int rpw = (int)(((int64_t)d->B * L.Nout + 8 * 148 * warps - 1) / (8 * 148 * warps));
-        rpw = rpw < 1 ? 1 : (rpw > 4 ? 4 : rpw);
-        const int copy_blocks = (L.Nout + warps * rpw - 1) / (warps * rpw);
-        dim3 grid(copy_blocks + L.S * L.colchunks, d->B);
-        hidden_merge_compact_kernel<<<grid, 256, 0, stream>>>(
-            static_cast<const uint4*>(hidden), static_cast<uint4*>(hidden_out), hid_sb / 8, out_sb / 8,
-            L.V, L.Nout, d->i0, d->n, d->k, src_map, d->N, wgt, meta, partial, L.S, L.colchunks,
-            copy_blocks, rpw);
-        if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
+        lvlm_status st;
+        const int chunks = (L.V + kHidThreads - 1) / kHidThreads;
+        if (chunks > kHidMaxChunks) return LVLM_ERR_UNSUPPORTED;       // more than 8192 channels
+        switch (chunks) {
+            case 1: st = launch_hidden_stream<1>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
+            case 2: st = launch_hidden_stream<2>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
+            case 3: st = launch_hidden_stream<3>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
+            case 4: st = launch_hidden_stream<4>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
+            default: return LVLM_ERR_UNSUPPORTED;
+        }
+        if (st != LVLM_OK) return st;
     } else {
         lvlm_status st = launch_inplace_compact(hidden, nullptr, hid_sb * 2, 0, d->B, 1, L.V,
                                                 L.Nout, src_map, wgt, meta, d->N, d->n, d->i0,
