@@ -219,7 +219,9 @@ class FullPass:
     @property
     def launches(self):
         w = self.w
-        return self.pre.launches + 2 * (w.L - self.first) + 2 + 2 * w.L
+        # reduction stages; 3 scoring kernels per compressed layer + plan and compaction; one decode
+        # kernel per layer
+        return self.pre.launches + 3 * (w.L - self.first) + 2 + w.L
 
 
 def bench_full(w, device, steps, warmup, flush, peaks, phases=True):
@@ -320,7 +322,7 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
            "decode_kv_bytes": bytes_read, "decode_gbs": bytes_read / (t_dec * 1e6),
            "decode_frac_hbm": bytes_read / (t_dec * 1e6) / peaks["hbm_gbs"],
            "compress_us_per_layer": (t_cmp * 1e3 / (n_cmp * w.L)) if n_cmp else None,
-           "final_len": cur_len, "launches": steps_total * 2 * w.L + n_cmp * 2}
+           "final_len": cur_len, "launches": steps_total * w.L + n_cmp * 2}
     if n_cmp:
         # bytes a compression must move per layer: read cap rows of K,V, write budget rows
         by = w.B * w.Hkv * ((w.budget + w.trigger) + w.budget) * 128 * 2 * 2
