@@ -31,6 +31,48 @@ inline lvlm_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? LVLM_OK : LVLM_ERR_CUDA;
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// Every kernel of the library is launched so that it may be scheduled while the kernel before it
+// in the stream is still draining (launch latency and the start-up of its CTAs overlap the tail
+// of that kernel).  The contract inside a kernel: pdl_wait() comes before the first access to
+// global memory that an earlier kernel may have written, or that an earlier kernel may still read
+// while this one writes it; once it returns, everything enqueued before is complete and visible.
+// pdl_launch_dependents() lets the next kernel start being scheduled; it comes right after the wait.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_launch_dependents(); }
+
+bool pdl_enabled();            // lvlm.cu; test hook lvlm_debug_set_pdl switches it off
+
+// Launches `kernel` with programmatic stream serialisation and, when cluster_x > 1, clusters of
+// cluster_x CTAs along x.
+template <typename... KArgs, typename... Args>
+inline lvlm_status launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, int cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (cluster_x > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)cluster_x;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl_enabled()) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess ? LVLM_OK : LVLM_ERR_CUDA;
+}
+
 // ---- bf16 <-> fp32 on packed words -------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

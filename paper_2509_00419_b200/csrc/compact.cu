@@ -55,6 +55,7 @@ __device__ __forceinline__ float ld_cluster_f32(const float* my_smem, uint32_t r
 // grid.x = column groups * S (clusters of S along x), grid.y = G (* 2 with a second tensor), grid.z = B
 __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const InplaceArgs a) {
     extern __shared__ __align__(16) uint4 tile[];
+    pdl_enter();
     const int S = a.S;
     const int rank = (int)cluster_rank();
     const int col = blockIdx.x / S;
@@ -263,20 +264,8 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
     if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(inplace_compact_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(ncol * S), (unsigned)(G * (base1 ? 2 : 1)), (unsigned)B);
-    cfg.blockDim = dim3(kCompactThreads, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)S;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, inplace_compact_kernel, a));
-    return LVLM_OK;
+    return launch_kernel(inplace_compact_kernel, dim3((unsigned)(ncol * S), (unsigned)(G * (base1 ? 2 : 1)), (unsigned)B),
+                         dim3(kCompactThreads), smem, stream, S, a);
 }
 
 }  // namespace lvlm

@@ -137,6 +137,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
     float* s_rm = s_FI + 8;                                             // [S][8] max of every CTA of the cluster
     float* s_rl = s_rm + 8 * kDecMaxCluster;                            // [S][8] sum of every CTA
 
+    pdl_enter();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.S, H = a.H, cap = a.cap;
     const int hd = blockIdx.x / S;
@@ -469,20 +470,7 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
     a.ws_s = acc_score ? reinterpret_cast<float*>(wsb + L.off_s) : nullptr;
     a.dev_status = dev_status;
 
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)ctas, 1, 1);
-    cfg.blockDim = dim3(kDecThreads, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)L.S;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, decode_cluster_kernel<G>, a));
-    return LVLM_OK;
+    return launch_kernel(decode_cluster_kernel<G>, dim3((unsigned)ctas), dim3(kDecThreads), smem, stream, L.S, a);
 }
 
 }  // namespace lvlm

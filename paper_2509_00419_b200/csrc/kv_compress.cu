@@ -93,6 +93,7 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
     __shared__ unsigned long long s_thr;
     __shared__ int s_below, s_first_drop;
 
+    pdl_enter();
     const int g = blockIdx.x, b = blockIdx.y;
     const int m_idx = b * Hkv + g;
     const int ln = len[m_idx];
@@ -223,10 +224,12 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
     const size_t smem = (size_t)P_max * 8 + (size_t)d->cap * 4;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(kv_plan_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    kv_plan_kernel<<<dim3(d->Hkv, d->B), threads, smem, stream>>>(
-        acc_score, pos, len, e_lo, e_hi, d->Hkv, d->cap, d->recent, P_max, beta_ppm, budget,
-        src_map, meta, nout, dev_status);
-    if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
+    {
+        const lvlm_status st = launch_kernel(kv_plan_kernel, dim3(d->Hkv, d->B), dim3(threads), smem, stream, 1,
+                                             acc_score, pos, len, e_lo, e_hi, d->Hkv, d->cap, d->recent, P_max,
+                                             beta_ppm, budget, src_map, meta, nout, dev_status);
+        if (st != LVLM_OK) return st;
+    }
     return launch_inplace_compact(Kc, Vc, kv_sb * 2, kv_sh * 2, d->B, d->Hkv, kHeadDim / 8, 0,
                                   src_map, nullptr, meta, d->cap, 0, 0, 0, 1, stream,
                                   /*maps_per_g=*/d->Hkv, /*map_stride=*/d->cap, nout);

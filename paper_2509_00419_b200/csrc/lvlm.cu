@@ -1,4 +1,6 @@
 // Version, status text and workspace sizes of the lvlm library.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace lvlm {
@@ -6,6 +8,17 @@ size_t score_tokens_workspace(const lvlm_dims* d);
 size_t merge_compact_workspace(const lvlm_dims* d);
 size_t kv_compress_workspace(const lvlm_dims* d);
 size_t decode_attn_workspace(const lvlm_dims* d);
+}  // namespace lvlm
+
+// Programmatic dependent launch of the library's kernels: on unless the environment variable
+// LVLM_NO_PDL is set or the test hook below switches it off.  Not part of the public header.
+static int g_pdl = -1;
+extern "C" void lvlm_debug_set_pdl(int on) { g_pdl = on ? 1 : 0; }
+namespace lvlm {
+bool pdl_enabled() {
+    if (g_pdl < 0) g_pdl = getenv("LVLM_NO_PDL") ? 0 : 1;
+    return g_pdl != 0;
+}
 }  // namespace lvlm
 
 extern "C" const char* lvlm_version(void) { return "lvlm 0.1 (sm_100a)"; }

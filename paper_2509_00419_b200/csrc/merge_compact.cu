@@ -91,6 +91,7 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
     __shared__ int scan_scratch[33];
     __shared__ float fsum_scratch[33];
     __shared__ int s_first_drop, s_merged_tok, s_pos_new;
+    pdl_enter();
     const int b = blockIdx.x;
     const int r1 = n - k, r = r1 - 1, Nout = N - r;
     const int32_t* rk = rank + (int64_t)b * n;
@@ -165,6 +166,7 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
 }
 
 __global__ void identity_len_kernel(int32_t* new_len, int B, int N) {
+    pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < B) new_len[b] = N;
 }
@@ -202,6 +204,7 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
                      int32_t* meta, float* partial) {
     extern __shared__ __align__(16) float s_sum[];           // [V][8] this CTA's sums
     __shared__ int s_last;
+    pdl_enter();
     const int b = blockIdx.y, cta = blockIdx.x, tid = threadIdx.x;
     const uint4* hin = hidden + (int64_t)b * hid_stride_b;
     uint4* hout = out + (int64_t)b * out_stride_b;
@@ -334,22 +337,10 @@ static lvlm_status launch_hidden_stream(const void* hidden, void* hidden_out, in
     const size_t smem = (size_t)L.V * 32;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(hidden_stream_kernel<CH>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)L.cps, (unsigned)d->B, 1);
-    cfg.blockDim = dim3(kHidThreads, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)L.cl;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, hidden_stream_kernel<CH>, static_cast<const uint4*>(hidden),
-                                           static_cast<uint4*>(hidden_out), hid_sb / 8, out_sb / 8, L.V, d->N,
-                                           d->i0, d->n, d->k, L.rpc, L.cl, dst_map, wgt, meta, partial));
-    return LVLM_OK;
+    return launch_kernel(hidden_stream_kernel<CH>, dim3((unsigned)L.cps, (unsigned)d->B), dim3(kHidThreads), smem,
+                         stream, L.cl, static_cast<const uint4*>(hidden), static_cast<uint4*>(hidden_out),
+                         hid_sb / 8, out_sb / 8, L.V, d->N, d->i0, d->n, d->k, L.rpc, L.cl, dst_map, wgt, meta,
+                         partial);
 }
 
 }  // namespace lvlm
@@ -388,8 +379,9 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
                                                   (size_t)d->N * d->C * 2, d->B,
                                                   cudaMemcpyDeviceToDevice, stream));
         }
-        if (new_len) identity_len_kernel<<<(d->B + 127) / 128, 128, 0, stream>>>(new_len, d->B, d->N);
-        return launch_status();
+        if (new_len) return launch_kernel(identity_len_kernel, dim3((d->B + 127) / 128), dim3(128), 0, stream, 1,
+                                          new_len, d->B, d->N);
+        return LVLM_OK;
     }
     if (!ws || !aligned256(ws) || ws_bytes < L.total) return LVLM_ERR_WORKSPACE;
     char* wsb = static_cast<char*>(ws);
@@ -403,10 +395,12 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     if (mode == LVLM_W_LINEAR_RANK) inv_sum = (float)(2.0 / ((double)L.r1 * ((double)L.r1 + 1.0)));
     else if (mode == LVLM_W_UNIFORM) inv_sum = (float)(1.0 / (double)L.r1);
     const int plan_threads = d->n >= 1024 ? 1024 : (d->n <= 128 ? 128 : ((d->n + 31) / 32) * 32);
-    merge_plan_kernel<<<d->B, plan_threads, 0, stream>>>(rank, pos_ids, d->N, d->i0, d->n, d->k,
-                                                         (int)mode, inv_sum, w_custom, src_map, dst_map,
-                                                         wgt, meta, new_len, dev_status);
-    if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
+    {
+        const lvlm_status st = launch_kernel(merge_plan_kernel, dim3(d->B), dim3(plan_threads), 0, stream, 1,
+                                             rank, pos_ids, d->N, d->i0, d->n, d->k, (int)mode, inv_sum, w_custom,
+                                             src_map, dst_map, wgt, meta, new_len, dev_status);
+        if (st != LVLM_OK) return st;
+    }
 
     if (hidden_out) {
         lvlm_status st;

@@ -44,6 +44,7 @@ score_colsum_simt_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     uint4* ktile = reinterpret_cast<uint4*>(colsum + ((n + 3) & ~3));   // [32 keys][16 vectors]
     float* wsum = reinterpret_cast<float*>(ktile + kRefKeys * 16);      // [4 warps][32 keys]
 
+    pdl_enter();
     const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int Nq = q_hi - q_lo;
@@ -143,6 +144,7 @@ __global__ void score_reduce_kernel(const float* __restrict__ partial, int P, in
                                     float inv_h, float* __restrict__ score,
                                     float* __restrict__ score_head, int64_t head_stride,
                                     int32_t* dev_status) {
+    pdl_enter();
     const int b = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
@@ -167,21 +169,19 @@ lvlm_status launch_score_simt(const void* Q, const void* K, const float* lse, co
     if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_colsum_simt_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    score_colsum_simt_kernel<<<dim3(d->H, d->B), kRefRows, smem, stream>>>(
-        static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K), lse, d->H,
-        d->H / d->Hkv, d->N, d->i0, d->n, d->q_lo, d->q_hi, d->causal, st.q_sb, st.q_sn, st.q_sh,
-        st.kv_sb, st.kv_sh, scale * kLog2eS, partial);
-    return launch_status();
+    return launch_kernel(score_colsum_simt_kernel, dim3(d->H, d->B), dim3(kRefRows), smem, stream, 1,
+                         static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K), lse, d->H,
+                         d->H / d->Hkv, d->N, d->i0, d->n, d->q_lo, d->q_hi, d->causal, st.q_sb, st.q_sn, st.q_sh,
+                         st.kv_sb, st.kv_sh, scale * kLog2eS, partial);
 }
 
 lvlm_status launch_score_reduce(const float* partial, bool group_summed, const lvlm_dims* d,
                                 float* score, float* score_head, int32_t* dev_status,
                                 cudaStream_t stream) {
-    score_reduce_kernel<<<dim3((d->n + 255) / 256, d->B), 256, 0, stream>>>(
-        partial, group_summed ? d->Hkv : d->H, group_summed ? 1 : d->H / d->Hkv, d->n,
-        1.0f / (float)d->H, score, score_head,
-        d->head_stride ? d->head_stride : (int64_t)d->n, dev_status);
-    return launch_status();
+    return launch_kernel(score_reduce_kernel, dim3((d->n + 255) / 256, d->B), dim3(256), 0, stream, 1,
+                         partial, group_summed ? d->Hkv : d->H, group_summed ? 1 : d->H / d->Hkv, d->n,
+                         1.0f / (float)d->H, score, score_head,
+                         d->head_stride ? d->head_stride : (int64_t)d->n, dev_status);
 }
 
 }  // namespace lvlm

@@ -96,6 +96,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
+    pdl_enter();                               // barriers and tensor memory are set up; now the inputs
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -261,13 +262,14 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
     if (!lse) {
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<0>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        score_tc_kernel<0><<<dim3(nqt, d->H, d->B), kTcThreads, smem, stream>>>(qmap, kmap, a);
-        if (cudaGetLastError() != cudaSuccess) return LVLM_ERR_CUDA;
+        const lvlm_status s0 = launch_kernel(score_tc_kernel<0>, dim3(nqt, d->H, d->B), dim3(kTcThreads), smem,
+                                             stream, 1, qmap, kmap, a);
+        if (s0 != LVLM_OK) return s0;
     }
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<1>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    score_tc_kernel<1><<<dim3(nkt, d->Hkv, d->B), kTcThreads, smem, stream>>>(qmap, kmap, a);
-    return launch_status();
+    return launch_kernel(score_tc_kernel<1>, dim3(nkt, d->Hkv, d->B), dim3(kTcThreads), smem, stream, 1,
+                         qmap, kmap, a);
 }
 
 }  // namespace lvlm

@@ -18,6 +18,7 @@ select_rank_kernel(const float* __restrict__ score, int64_t stride, int n, int k
     __shared__ int scan_scratch[33];
     __shared__ int s_near;
 
+    pdl_enter();
     const int b = blockIdx.x;
     const float* row = score + (int64_t)b * stride;
     bool nonfinite = false;
@@ -82,7 +83,6 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
     const size_t smem = (size_t)P * 8 + (size_t)n * 4;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_rank_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    select_rank_kernel<<<B, threads, smem, (cudaStream_t)stream>>>(
-        score, score_stride, n, k, P, rank, kept_idx, near_tie, dev_status);
-    return launch_status();
+    return launch_kernel(select_rank_kernel, dim3(B), dim3(threads), smem, (cudaStream_t)stream, 1,
+                         score, score_stride, n, k, P, rank, kept_idx, near_tie, dev_status);
 }
