@@ -21,6 +21,7 @@ bool score_layout(const lvlm_dims* d, ScoreLayout* L) {
     size_t off = 0;
     L->off_partial = off; off = align_up(off + (size_t)d->B * d->H * d->n * 4, 256);
     L->off_lse = off;     off = align_up(off + (size_t)d->B * d->H * (d->q_hi - d->q_lo) * 4, 256);
+    L->off_cnt = off;     off = align_up(off + (size_t)d->B * ((d->n + 127) / 128) * 4, 256);
     L->total = off;
     return true;
 }
@@ -220,7 +221,6 @@ extern "C" lvlm_status lvlm_score_tokens(const void* Q, const void* K, const flo
         return launch_score_reduce(partial, false, d, score, score_head, dev_status, stream);
     }
     float* lse_ws = reinterpret_cast<float*>(wsb + L.off_lse);
-    lvlm_status s = launch_score_tc(Q, K, lse, d, st, scale, lse_ws, partial, dev_status, stream);
-    if (s != LVLM_OK) return s;
-    return launch_score_reduce(partial, true, d, score, score_head, dev_status, stream);
+    return launch_score_tc(Q, K, lse, d, st, scale, lse_ws, partial,
+                           reinterpret_cast<int32_t*>(wsb + L.off_cnt), score, score_head, dev_status, stream);
 }

@@ -4,7 +4,7 @@
 
 namespace lvlm {
 
-struct ScoreLayout { size_t off_partial, off_lse, total; };
+struct ScoreLayout { size_t off_partial, off_lse, off_cnt, total; };
 struct ScoreStrides { int64_t q_sb, q_sn, q_sh, kv_sb, kv_sh; };   // elements
 
 bool score_layout(const lvlm_dims* d, ScoreLayout* L);
@@ -14,9 +14,11 @@ lvlm_status launch_score_reduce(const float* partial, bool group_summed, const l
                                 cudaStream_t stream);
 
 // Tensor-core path: pass 1 (row normalisers into lse_ws, skipped when the caller supplies lse) and
-// pass 2 (group-summed column sums into partial [B][Hkv][n]).
+// pass 2 (column sums per CTA row into partial, added over the heads by the last CTA of each key
+// tile, which writes score and score_head).  cnt holds one counter per (sequence, key tile).
 lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, const lvlm_dims* d,
                             const ScoreStrides& st, float scale, float* lse_ws, float* partial,
-                            int32_t* dev_status, cudaStream_t stream);
+                            int32_t* cnt, float* score, float* score_head, int32_t* dev_status,
+                            cudaStream_t stream);
 
 }  // namespace lvlm

@@ -32,7 +32,13 @@ struct ScoreTcArgs {
     float scale_log2;
     const float* lse_user;     // natural-log row normalisers from the caller, or NULL
     float* lse_ws;             // [B][H][Nq] log2-domain normalisers (pass 1 writes, pass 2 reads)
-    float* partial;            // [B][Hkv][n] group-summed column sums (pass 2 writes)
+    float* partial;            // [B][Hkv * hsplit][n] column sums of each CTA row (pass 2 writes)
+    int nkt;                   // key tiles of pass 2 (its grid.x)
+    int hsplit;                // CTAs that share the query heads of one KV group in pass 2
+    int32_t* cnt;              // [B][key tiles] CTAs of pass 2 that have parked their sums (zero at its start)
+    float* score;              // [B][n] head mean (written by the last CTA of a key tile)
+    float* score_head;         // optional [B][Hkv] rows of n, head_stride apart
+    int64_t head_stride;
     int32_t* dev_status;
 };
 
@@ -40,6 +46,7 @@ struct TcSmem {
     uint64_t a_full, full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort;
+    volatile int last;
     float lse_s[4][2][kTile];      // per epilogue warp, per accumulator buffer
 };
 
@@ -68,17 +75,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
 
     // ---- which tiles this CTA multiplies ---------------------------------------------------------
     int nt, h = 0, g = 0, qt = 0, kt = 0, qt_min = 0, nqt_vis = 0;
+    const int h_first = MODE == 1 ? (blockIdx.y / a.hsplit) * a.G + (blockIdx.y % a.hsplit) * (a.G / a.hsplit) : 0;
     if (MODE == 0) {
         qt = blockIdx.x; h = blockIdx.y; g = h / a.G;
         const int last_pos = a.q_lo + min(a.Nq, (qt + 1) * kTile) - 1;
         const int key_end = a.causal ? min(a.N, last_pos + 1) : a.N;
         nt = (key_end + kTile - 1) / kTile;
     } else {
-        kt = blockIdx.x; g = blockIdx.y;
+        kt = blockIdx.x; g = blockIdx.y / a.hsplit;
         const int j0 = a.i0 + kt * kTile;
         qt_min = a.causal ? max(0, (j0 - a.q_lo) / kTile) : 0;
         nqt_vis = max(0, nqt - qt_min);
-        nt = a.G * nqt_vis;
+        nt = (a.G / a.hsplit) * nqt_vis;
     }
 
     if (threadIdx.x == 0) {
@@ -97,6 +105,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
     pdl_enter();                               // barriers and tensor memory are set up; now the inputs
+    if (MODE == 0 && blockIdx.x == 0 && blockIdx.y == 0)      // pass 2 counts its CTAs per key tile from zero
+        for (int i = threadIdx.x; i < a.nkt; i += blockDim.x) a.cnt[b * a.nkt + i] = 0;
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -118,7 +128,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
                     tma_load_4d(dst, &kmap, &sm->full[st], 0, t * kTile, g, b);
                     tma_load_4d(dst + kHalfBytes, &kmap, &sm->full[st], 64, t * kTile, g, b);
                 } else {
-                    const int hh = g * a.G + t / nqt_vis, q2 = qt_min + t % nqt_vis;
+                    const int hh = h_first + t / nqt_vis, q2 = qt_min + t % nqt_vis;
                     tma_load_4d(dst, &qmap, &sm->full[st], 0, hh, q2 * kTile, b);
                     tma_load_4d(dst + kHalfBytes, &qmap, &sm->full[st], 64, hh, q2 * kTile, b);
                 }
@@ -156,23 +166,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
         float m_run = -INFINITY, l_run = 0.f, colsum = 0.f;
         const int my_pos = a.q_lo + qt * kTile + row;        // MODE 0: sequence position of my query
         const int my_key = a.i0 + kt * kTile + row;          // MODE 1: my key
+        // row normalisers of a tile (MODE 1): every warp keeps its own copy of the tile's 128 values;
+        // they are fetched one tile ahead so that the loads never sit on the critical path
+        float lse_next[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
+        auto fetch_lse = [&](int t) {
+            const int hh = h_first + t / nqt_vis, q2l = qt_min + t % nqt_vis;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = q2l * kTile + u * 32 + lane;
+                float v = INFINITY;                            // rows past the window add nothing
+                if (i < a.Nq) {
+                    const int64_t idx = ((int64_t)b * a.H + hh) * a.Nq + i;
+                    v = a.lse_user ? a.lse_user[idx] * kLog2eT : __ldcg(a.lse_ws + idx);
+                }
+                lse_next[u] = v;
+            }
+        };
+        if (MODE == 1 && nt > 0) fetch_lse(0);
         for (int t = 0; t < nt; ++t) {
             const int buf = t & 1;
             int q2 = 0;
             if (MODE == 1) {
-                const int hh = g * a.G + t / nqt_vis;
                 q2 = qt_min + t % nqt_vis;
-                // every warp stages its own copy of the tile's 128 row normalisers (no block barrier)
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = q2 * kTile + u * 32 + lane;
-                    float v = INFINITY;                        // rows past the window add nothing
-                    if (i < a.Nq) {
-                        const int64_t idx = ((int64_t)b * a.H + hh) * a.Nq + i;
-                        v = a.lse_user ? a.lse_user[idx] * kLog2eT : a.lse_ws[idx];
-                    }
-                    sm->lse_s[warp - 2][buf][u * 32 + lane] = v;
-                }
+                for (int u = 0; u < 4; ++u) sm->lse_s[warp - 2][buf][u * 32 + lane] = lse_next[u];
+                if (t + 1 < nt) fetch_lse(t + 1);
                 __syncwarp();
             }
             if (!wait_or_abort(&sm->tmem_full[buf], (t / 2) & 1, sm, a.dev_status)) break;
@@ -214,13 +232,37 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
             tc_fence_before();
             mbar_arrive(&sm->tmem_empty[buf]);
         }
-        if (!sm->abort) {
-            if (MODE == 0) {
-                const int i = qt * kTile + row;
-                if (i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = m_run + log2f(l_run);
-            } else {
-                const int jl = kt * kTile + row;
-                if (jl < a.n) a.partial[((int64_t)b * (a.H / a.G) + g) * a.n + jl] = colsum;
+        if (MODE == 0) {
+            const int i = qt * kTile + row;
+            if (!sm->abort && i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = m_run + log2f(l_run);
+        } else {
+            // every epilogue thread takes this path, also after a timeout, so that the counters and
+            // the barriers below always see all 128 of them
+            const int Hkv = a.H / a.G, P = Hkv * a.hsplit;       // CTA rows per sequence
+            const int jl = kt * kTile + row;
+            if (jl < a.n) a.partial[((int64_t)b * P + blockIdx.y) * a.n + jl] = colsum;
+            // the last CTA of this key tile adds the rows in row order: head mean and group sums
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) sm->last = atomicAdd(&a.cnt[b * gridDim.x + kt], 1) == P - 1;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (sm->last) {
+                __threadfence();
+                if (jl < a.n) {
+                    float tot = 0.f;
+                    for (int gg = 0; gg < Hkv; ++gg) {
+                        float gs = 0.f;
+                        for (int pp = 0; pp < a.hsplit; ++pp)
+                            gs += __ldcg(a.partial + ((int64_t)b * P + gg * a.hsplit + pp) * a.n + jl);
+                        if (a.score_head) a.score_head[((int64_t)b * Hkv + gg) * a.head_stride + jl] = gs;
+                        tot += gs;
+                    }
+                    const float sc = tot * (1.0f / (float)a.H);
+                    a.score[(int64_t)b * a.n + jl] = sc;
+                    if (a.dev_status && (__float_as_uint(sc) & 0x7F800000u) == 0x7F800000u)
+                        atomicOr(a.dev_status, LVLM_DEV_NONFINITE);
+                }
+                if (threadIdx.x == 64) a.cnt[b * gridDim.x + kt] = 0;
             }
         }
     }
@@ -238,7 +280,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
 
 lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, const lvlm_dims* d,
                             const ScoreStrides& st, float scale, float* lse_ws, float* partial,
-                            int32_t* dev_status, cudaStream_t stream) {
+                            int32_t* cnt, float* score, float* score_head, int32_t* dev_status,
+                            cudaStream_t stream) {
     const int Nq = d->q_hi - d->q_lo;
     CUtensorMap qmap, kmap;
     {
@@ -257,8 +300,20 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
     a.B = d->B; a.H = d->H; a.G = d->H / d->Hkv; a.N = d->N; a.Nq = Nq; a.i0 = d->i0; a.n = d->n;
     a.q_lo = d->q_lo; a.causal = d->causal; a.scale_log2 = scale * kLog2eT;
     a.lse_user = lse; a.lse_ws = lse_ws; a.partial = partial; a.dev_status = dev_status;
+    a.cnt = cnt; a.score = score; a.score_head = score_head;
+    a.head_stride = d->head_stride ? d->head_stride : (int64_t)d->n;
     const size_t smem = 1024 + (size_t)kTileBytes * (1 + kStages) + sizeof(TcSmem);
     const int nqt = (Nq + kTile - 1) / kTile, nkt = (d->n + kTile - 1) / kTile;
+    // pass 2: when key tiles x KV heads do not fill the GPU, the query heads of a group are shared
+    // out over several CTAs (the smallest divisor of G that gets there, else all of G)
+    int hsplit = 1;
+    for (int hs = 1; hs <= a.G; ++hs) {
+        if (a.G % hs) continue;
+        hsplit = hs;
+        if ((int64_t)nkt * d->Hkv * d->B * hs >= 148) break;
+    }
+    a.hsplit = hsplit; a.nkt = nkt;
+    if (lse) LVLM_RETURN_IF_CUDA(cudaMemsetAsync(cnt, 0, (size_t)d->B * nkt * 4, stream));
     if (!lse) {
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<0>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -268,7 +323,7 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
     }
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<1>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    return launch_kernel(score_tc_kernel<1>, dim3(nkt, d->Hkv, d->B), dim3(kTcThreads), smem, stream, 1,
+    return launch_kernel(score_tc_kernel<1>, dim3(nkt, d->Hkv * hsplit, d->B), dim3(kTcThreads), smem, stream, 1,
                          qmap, kmap, a);
 }
 
