@@ -23,7 +23,8 @@ constexpr int kTile = 128;                 // rows of A, rows of B, and K (= hea
 constexpr int kStages = 4;                 // B-tile ring
 constexpr int kHalfBytes = kTile * 64 * 2; // one TMA box: 128 rows x 64 bf16 = 16 KB
 constexpr int kTileBytes = 2 * kHalfBytes; // 32 KB
-constexpr int kTcThreads = 192;            // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kTcThreads = 320;            // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kEpiThreads = 256;           // two warps per quarter of the TMEM lanes, 64 columns each
 constexpr uint32_t kTmemCols = 256;        // two 128-column fp32 accumulators
 constexpr float kLog2eT = 1.4426950408889634f;
 
@@ -47,7 +48,8 @@ struct TcSmem {
     uint32_t tmem_base;
     volatile int abort;
     volatile int last;
-    float lse_s[4][2][kTile];      // per epilogue warp, per accumulator buffer
+    float lse_s[8][2][kTile / 2];  // per epilogue warp, per accumulator buffer: normalisers of its 64 columns
+    float xm[kTile], xl[kTile];    // what the warps of the upper column half hand to the lower half
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, TcSmem* sm, int32_t* dev_status) {
@@ -92,7 +94,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     if (threadIdx.x == 0) {
         mbar_init(&sm->a_full, 1);
         for (int s = 0; s < kStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sm->tmem_full[s], 1); mbar_init(&sm->tmem_empty[s], 128); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sm->tmem_full[s], 1); mbar_init(&sm->tmem_empty[s], kEpiThreads); }
         sm->abort = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -159,8 +161,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
             }
         }
     } else {
-        // ================= epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 =================
-        const int quarter = warp & 3;
+        // ===== epilogue: warps 2..9; a warp reads TMEM lanes 32*(warp%4) .. +31, columns 64*half .. +63 =====
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;                 // TMEM lane = row of the A tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
         float m_run = -INFINITY, l_run = 0.f, colsum = 0.f;
@@ -168,12 +170,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
         const int my_key = a.i0 + kt * kTile + row;          // MODE 1: my key
         // row normalisers of a tile (MODE 1): every warp keeps its own copy of the tile's 128 values;
         // they are fetched one tile ahead so that the loads never sit on the critical path
-        float lse_next[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
+        float lse_next[2] = {INFINITY, INFINITY};
         auto fetch_lse = [&](int t) {
             const int hh = h_first + t / nqt_vis, q2l = qt_min + t % nqt_vis;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = q2l * kTile + u * 32 + lane;
+            for (int u = 0; u < 2; ++u) {
+                const int i = q2l * kTile + half * 64 + u * 32 + lane;
                 float v = INFINITY;                            // rows past the window add nothing
                 if (i < a.Nq) {
                     const int64_t idx = ((int64_t)b * a.H + hh) * a.Nq + i;
@@ -189,14 +191,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
             if (MODE == 1) {
                 q2 = qt_min + t % nqt_vis;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) sm->lse_s[warp - 2][buf][u * 32 + lane] = lse_next[u];
+                for (int u = 0; u < 2; ++u) sm->lse_s[warp - 2][buf][u * 32 + lane] = lse_next[u];
                 if (t + 1 < nt) fetch_lse(t + 1);
                 __syncwarp();
             }
             if (!wait_or_abort(&sm->tmem_full[buf], (t / 2) & 1, sm, a.dev_status)) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
+            for (int c2 = 0; c2 < 2; ++c2) {
+                const int c4 = half * 2 + c2;                  // 32-column chunk of the tile
                 float v[32];
                 tmem_ld32(lane_addr + buf * kTile + c4 * 32, v);
                 tmem_ld_wait();
@@ -221,7 +224,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
                     const int ib = q2 * kTile + c4 * 32;                           // first query row of the chunk
                     // query i sees my key iff my_key <= q_lo + i  <=>  c >= my_key - q_lo - ib
                     const int first = a.causal ? my_key - a.q_lo - ib : 0;
-                    const float* ls = &sm->lse_s[warp - 2][buf][c4 * 32];
+                    const float* ls = &sm->lse_s[warp - 2][buf][c2 * 32];
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
                         const float p = exp2f(v[c] * a.scale_log2 - ls[c]);
@@ -232,21 +235,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
             tc_fence_before();
             mbar_arrive(&sm->tmem_empty[buf]);
         }
+        // the two column halves of a row meet in shared memory; every epilogue thread takes this path,
+        // also after a timeout, so that the barriers and the counters always see all of them
+        if (half == 1) { sm->xm[row] = MODE == 0 ? m_run : colsum; sm->xl[row] = l_run; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (MODE == 0) {
-            const int i = qt * kTile + row;
-            if (!sm->abort && i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = m_run + log2f(l_run);
+            if (half == 0) {
+                const float m1 = sm->xm[row], l1 = sm->xl[row];
+                const float M = fmaxf(m_run, m1);
+                float L = 0.f;
+                if (m_run > -INFINITY) L += l_run * exp2f(m_run - M);
+                if (m1 > -INFINITY) L += l1 * exp2f(m1 - M);
+                const int i = qt * kTile + row;
+                if (!sm->abort && i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = M + log2f(L);
+            }
         } else {
-            // every epilogue thread takes this path, also after a timeout, so that the counters and
-            // the barriers below always see all 128 of them
+            if (half == 0) colsum += sm->xm[row];
             const int Hkv = a.H / a.G, P = Hkv * a.hsplit;       // CTA rows per sequence
             const int jl = kt * kTile + row;
-            if (jl < a.n) a.partial[((int64_t)b * P + blockIdx.y) * a.n + jl] = colsum;
+            if (half == 0 && jl < a.n) a.partial[((int64_t)b * P + blockIdx.y) * a.n + jl] = colsum;
             // the last CTA of this key tile adds the rows in row order: head mean and group sums
             __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (threadIdx.x == 64) sm->last = atomicAdd(&a.cnt[b * gridDim.x + kt], 1) == P - 1;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (sm->last) {
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (sm->last && half == 0) {
                 __threadfence();
                 if (jl < a.n) {
                     float tot = 0.f;
