@@ -20,7 +20,7 @@ namespace lvlm {
 using namespace sm100;
 
 constexpr int kTile = 128;                 // rows of A, rows of B, and K (= head dim)
-constexpr int kStages = 4;                 // B-tile ring
+constexpr int kStages = 2;                 // B-tile ring (two CTAs fit on an SM)
 constexpr int kHalfBytes = kTile * 64 * 2; // one TMA box: 128 rows x 64 bf16 = 16 KB
 constexpr int kTileBytes = 2 * kHalfBytes; // 32 KB
 constexpr int kTcThreads = 320;            // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
@@ -61,7 +61,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Tc
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
                 const ScoreTcArgs a) {
     extern __shared__ unsigned char smem_dyn[];
