@@ -17,7 +17,7 @@ class ReduceStage:
     """score_tokens -> select_topk -> merge_compact for one layer (Section 3.2.1), with every
     output and workspace allocated once so that the calls can be captured in a CUDA graph."""
 
-    LAUNCHES = 3 + 1 + 3      # score (normalisers, column sums, head reduction), select,
+    LAUNCHES = 2 + 1 + 3      # score (normalisers, column sums + head reduction), select,
                               # merge_compact (plan, hidden, K/V)
 
     def __init__(self, B, N, C, H, Hkv, cap, i0, n, M, device, want_head=False, mode=L.W_LINEAR_RANK):
