@@ -242,23 +242,40 @@ def merge_compact(hidden, rank, i0, n, k, mode=LINEAR_RANK, custom=None,
     return out
 
 
-def nearest_kept_merge(hidden, rank, i0, n, k, mass=None):
+def nearest_kept_merge(hidden, rank, i0, n, k, mass=None, Kc=None, Vc=None, pos_ids=None, assign=None):
     """North-star variant (not in the paper): every dropped image token is merged into
     the kept image token it is most similar to.
 
     For a dropped token d (rank >= k): a(d) = argmax over kept t of the cosine
-    similarity of rows d and t (lower t wins ties).  Each kept t becomes the
-    mass-weighted mean of itself and the tokens assigned to it; masses default to 1.
-    Output has the k kept image tokens only (no extra row): length N - (n - k).
+    similarity of the hidden rows d and t (lower t wins ties).  Each kept t becomes the
+    mass-weighted mean of itself and the tokens assigned to it, added in ascending
+    token order; masses default to 1.  Output has the k kept image tokens only (no
+    extra row): length N - (n - k).  That layer's Kc, Vc [B, Hkv, N, D] follow the same
+    assignment and masses per KV head; pos_ids [B, N] keep the kept tokens' ids.
+    ``assign`` [B, n-k], when given, replaces the argmax (a test that has verified a
+    near-tie continues from the other side's choice).
     Returns dict(hidden, assign [B, n-k] (index into the ascending kept list, dropped
-    tokens in ascending index order), mass [B, N-(n-k)] or None, new_len).
+    tokens in ascending index order), sim_best / sim_second [B, n-k] (cosine of the
+    chosen and of the runner-up kept token), mass [B, N-(n-k)] or None, Kc, Vc,
+    pos_ids, new_len).
     """
     hidden = np.asarray(hidden, dtype=np.float64)
     B, N, C = hidden.shape
     r = n - k
     h_out = np.zeros((B, N - r, C), dtype=np.float32)
-    assign = np.zeros((B, r), dtype=np.int32)
+    a_out = np.zeros((B, r), dtype=np.int32)
+    best = np.zeros((B, r), dtype=np.float64)
+    second = np.full((B, r), -np.inf, dtype=np.float64)
     m_out = None if mass is None else np.zeros((B, N - r), dtype=np.float32)
+    K_out = V_out = p_out = None
+    if Kc is not None:
+        Kc = np.asarray(Kc, dtype=np.float64)
+        Vc = np.asarray(Vc, dtype=np.float64)
+        K_out = np.zeros((B, Kc.shape[1], N - r, Kc.shape[3]), dtype=np.float32)
+        V_out = np.zeros_like(K_out)
+    if pos_ids is not None:
+        pos_ids = np.asarray(pos_ids, dtype=np.int32)
+        p_out = np.zeros((B, N - r), dtype=np.int32)
     for b in range(B):
         rk = np.asarray(rank[b])
         kept = np.nonzero(rk < k)[0]
@@ -267,21 +284,36 @@ def nearest_kept_merge(hidden, rank, i0, n, k, mass=None):
         nrm = np.sqrt((x * x).sum(axis=1))
         nrm = np.where(nrm > 0, nrm, 1.0)
         m = np.ones(n) if mass is None else np.asarray(mass[b, i0:i0 + n], dtype=np.float64)
-        num = x[kept] * m[kept, None]
         den = m[kept].copy()
         for q, d in enumerate(drop):
-            cos = (x[kept] @ x[d]) / (nrm[kept] * nrm[d])
-            t = int(np.argmax(cos))                         # first maximum = lowest index
-            assign[b, q] = t
-            num[t] += m[d] * x[d]
+            cos = (x[kept] @ x[d]) / (nrm[kept] * nrm[d]) if k > 0 else np.zeros(0)
+            t = int(np.argmax(cos)) if assign is None else int(assign[b][q])   # first maximum = lowest index
+            a_out[b, q] = t
+            best[b, q] = cos[t]
+            if k > 1:
+                second[b, q] = np.max(np.delete(cos, t))
             den[t] += m[d]
-        img = num / den[:, None]
-        h_out[b] = round_bf16(np.concatenate([hidden[b, :i0], img, hidden[b, i0 + n:]], axis=0))
+
+        def merged(rows):                                   # rows [n, width] float64 -> [k, width]
+            num = rows[kept] * m[kept, None]
+            for q, d in enumerate(drop):
+                num[a_out[b, q]] += m[d] * rows[d]
+            return num / den[:, None]
+
+        h_out[b] = round_bf16(np.concatenate([hidden[b, :i0], merged(x), hidden[b, i0 + n:]], axis=0))
+        if Kc is not None:
+            for g in range(Kc.shape[1]):
+                K_out[b, g] = round_bf16(np.concatenate(
+                    [Kc[b, g, :i0], merged(Kc[b, g, i0:i0 + n]), Kc[b, g, i0 + n:N]], axis=0))
+                V_out[b, g] = round_bf16(np.concatenate(
+                    [Vc[b, g, :i0], merged(Vc[b, g, i0:i0 + n]), Vc[b, g, i0 + n:N]], axis=0))
+        if pos_ids is not None:
+            p_out[b] = np.concatenate([pos_ids[b, :i0], pos_ids[b, i0 + kept], pos_ids[b, i0 + n:]])
         if mass is not None:
             mm = np.asarray(mass[b], dtype=np.float64)
             m_out[b] = np.concatenate([mm[:i0], den, mm[i0 + n:]]).astype(np.float32)
-    return {"hidden": h_out, "assign": assign, "mass": m_out,
-            "new_len": np.full(B, N - r, dtype=np.int32)}
+    return {"hidden": h_out, "assign": a_out, "sim_best": best, "sim_second": second, "mass": m_out,
+            "Kc": K_out, "Vc": V_out, "pos_ids": p_out, "new_len": np.full(B, N - r, dtype=np.int32)}
 
 
 # ----------------------------------------------------------------------------

@@ -298,6 +298,18 @@ def test_nearest_kept_bruteforce_and_mass_conservation():
     tot_in = x.sum(axis=0)
     tot_out = (out["hidden"][0, i0:i0 + k].astype(np.float64) * out["mass"][0, i0:i0 + k, None]).sum(axis=0)
     np.testing.assert_allclose(tot_out, tot_in, atol=0.1)
+    # K, V and the position ids follow the same assignment: a cache that equals the hidden states
+    # comes out equal to them; a forced assignment is obeyed; the runner-up is never more similar
+    pos = np.arange(N, dtype=np.int32)[None]
+    kv = O.nearest_kept_merge(hidden, rank, i0, n, k, mass=mass, Kc=hidden[:, None], Vc=2 * hidden[:, None], pos_ids=pos)
+    np.testing.assert_array_equal(kv["Kc"][0, 0], out["hidden"][0])
+    np.testing.assert_array_equal(kv["Vc"][0, 0], O.round_bf16(2 * out["hidden"][0].astype(np.float64)))
+    np.testing.assert_array_equal(kv["pos_ids"][0], np.concatenate([pos[0, :i0], i0 + kept[0], pos[0, i0 + n:]]))
+    assert (out["sim_best"] >= out["sim_second"]).all()
+    forced = np.zeros_like(out["assign"])
+    f = O.nearest_kept_merge(hidden, rank, i0, n, k, assign=forced)
+    assert (f["assign"] == 0).all() and f["mass"] is None
+    np.testing.assert_array_equal(f["hidden"][0, i0], O.round_bf16((x[kept[0][0]] + x[drop].sum(axis=0)) / (1 + len(drop))))
 
 
 # ------------------------------------------------------------------ kv compression
