@@ -54,7 +54,13 @@ enum { LVLM_DEV_NONFINITE = 1, LVLM_DEV_TIMEOUT = 2, LVLM_DEV_BOUNDS = 4 };
  *   UNIFORM       1/(r+1) each
  *   CUSTOM        caller-supplied list w_custom[0..r]
  *   NEAREST_KEPT  not in the paper: each dropped token is averaged into the kept token with
- *                 the highest cosine similarity (lower index wins ties); no extra token */
+ *                 the highest cosine similarity of the hidden rows (lower index wins ties),
+ *                 weighted by the token masses; that layer's K and V rows are averaged with
+ *                 the same assignment; no extra token.  Needs hidden_out (out of place),
+ *                 1 <= k, n - k <= 16384, and a workspace sized with d->merge_mode set to it.
+ *                 After the call the first B*(n-k) int32 of `ws` hold the assignment: for the
+ *                 dropped tokens in ascending order, the index of their kept token in the
+ *                 ascending list of kept tokens. */
 typedef enum {
     LVLM_W_LINEAR_RANK = 0, LVLM_W_GEOMETRIC = 1, LVLM_W_UNIFORM = 2,
     LVLM_W_CUSTOM = 3, LVLM_W_NEAREST_KEPT = 4
@@ -82,6 +88,7 @@ typedef struct lvlm_dims {
     int32_t q_hi;     /* scoring: one past the last query row of the window */
     int32_t causal;   /* scoring: 1 = row at position p sees keys j <= p; 0 = sees all N keys */
     int32_t recent;   /* kv_compress: this many newest entries of every head are never evicted */
+    int32_t merge_mode; /* lvlm_workspace_bytes(LVLM_OP_MERGE_COMPACT): the lvlm_merge_mode to size for */
     int64_t q_stride_b, q_stride_n, q_stride_h;  /* Q[b][i][h][D]; default packed [B][q_hi-q_lo][H][D] */
     int64_t kv_stride_b, kv_stride_h;            /* K,V[b][g][row][D], rows packed; default [B][Hkv][cap][D] */
     int64_t hid_stride_b;                        /* hidden[b][row][C], rows packed; default N*C */
@@ -157,7 +164,8 @@ lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_str
  *               important merged token
  *   rank        [B][n] int32 from lvlm_select_topk (must be a permutation of 0..n-1)
  *   w_custom    [n-k] fp32 (device) when mode == CUSTOM, else NULL
- *   mass        NEAREST_KEPT only, optional [B][N] fp32 in/out: token masses (NULL = all 1)
+ *   mass        NEAREST_KEPT only, optional [B][N] fp32 in/out: token masses (NULL = all 1),
+ *               compacted in place like pos_ids; a kept token's mass grows by what it absorbs
  *   new_len     optional [B] int32 out: rows after the call
  * Reads d: B,N,C,Hkv,D,cap,i0,n,k,hid_stride_b,out_stride_b,kv_stride_*.
  * Errors: INVALID_ARG (NULL hidden/rank, i0+n>N, k outside [0,n], N>cap with Kc, only one of

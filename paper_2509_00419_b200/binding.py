@@ -31,7 +31,7 @@ class Dims(ctypes.Structure):
     """Mirror of ``lvlm_dims``."""
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "H", "Hkv", "D", "N", "C", "cap", "i0", "n", "k", "q_lo", "q_hi", "causal",
-                 "recent")] + \
+                 "recent", "merge_mode")] + \
                [(n, ctypes.c_int64) for n in
                 ("q_stride_b", "q_stride_n", "q_stride_h", "kv_stride_b", "kv_stride_h",
                  "hid_stride_b", "out_stride_b", "head_stride")]
@@ -204,6 +204,7 @@ def merge_compact(hidden, rank, *, i0, k, mode=W_LINEAR_RANK, Kc=None, Vc=None, 
     B, N, C = hidden.shape
     n = rank.shape[1]
     d = merge_dims(hidden, rank, i0=i0, k=k, Kc=Kc)
+    d.merge_mode = int(mode)
     rows = merged_rows(N, n, k, mode)
     if in_place:
         out = None
@@ -219,6 +220,12 @@ def merge_compact(hidden, rank, *, i0, k, mode=W_LINEAR_RANK, Kc=None, Vc=None, 
                                     _ptr(mass), _ptr(new_len), wsp, wsn, _ptr(dev_status),
                                     _stream(stream)), "lvlm_merge_compact")
     return (hidden if in_place else out), new_len
+
+
+def nearest_assignment(ws: torch.Tensor, B: int, r: int) -> torch.Tensor:
+    """Assignment lvlm_merge_compact leaves at the start of its workspace in mode NEAREST_KEPT:
+    [B, r] int32, for the dropped tokens in ascending order the index of their kept token."""
+    return ws[:B * r * 4].view(torch.int32).view(B, r)
 
 
 def kv_dims(Kc, *, H=None, recent=0) -> Dims:

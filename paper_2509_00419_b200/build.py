@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liblvlm.so")
 SOURCES = ["lvlm.cu", "select.cu", "compact.cu", "merge_compact.cu", "kv_compress.cu",
-           "decode.cu", "score.cu", "score_tc.cu"]
+           "decode.cu", "score.cu", "score_tc.cu", "nearest_kept.cu"]
 
 
 def _nvcc() -> str:

@@ -8,18 +8,35 @@
 // kept and adds it to the weighted sum if it is merged; (3) one kernel compacts K and V in place.
 #include "common.cuh"
 #include "compact.cuh"
+#include "merge.cuh"
 
 namespace lvlm {
 
 struct MergeLayout {
-    int r1, r, Nout, V, cps, cl, rpc;      // CTAs per sequence, cluster size, input rows per CTA
+    int r1, r, Nout, V;
+    HiddenGrid grid;
     size_t off_src, off_dst, off_wgt, off_meta, off_partial, total;
 };
 
 constexpr int kHidThreads = 256;       // streaming kernel: thread = 16-byte column group (+256, +512 ...)
 constexpr int kHidMaxChunks = 4;       // column groups per thread: rows up to 4 * 256 * 8 = 8192 channels
+constexpr int kNoRow = -2147483647 - 1;  // marks a slot of the four-row group that lies past the CTA's rows
 constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
-constexpr int kMetaInts = 4;           // per sequence: first moved row, ticket counter, merged token, spare
+
+// One wave of four CTAs per SM over the whole batch, at least 8 input rows each; clusters of 8.
+HiddenGrid hidden_grid(const lvlm_dims* d) {
+    HiddenGrid g;
+    g.V = d->C / 8;
+    int cps = (4 * 148) / d->B;
+    const int max_by_rows = (d->N + 7) / 8;
+    cps = cps > max_by_rows ? max_by_rows : cps;
+    cps = cps < 1 ? 1 : cps;
+    g.cl = cps >= kHidCluster ? kHidCluster : 1;
+    cps = cps / g.cl * g.cl;
+    g.cps = cps;
+    g.rpc = (d->N + cps - 1) / cps;
+    return g;
+}
 
 static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
     if (!d || d->B <= 0 || d->N <= 0 || d->n <= 0 || d->C <= 0 || d->C % 8 || d->i0 < 0 ||
@@ -29,26 +46,20 @@ static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
     L->r = L->r1 > 0 ? L->r1 - 1 : 0;
     L->Nout = d->N - L->r;
     L->V = d->C / 8;
-    // one wave of four CTAs per SM over the whole batch, at least 8 input rows each
-    int cps = (4 * 148) / d->B;
-    const int max_by_rows = (d->N + 7) / 8;
-    cps = cps > max_by_rows ? max_by_rows : cps;
-    cps = cps < 1 ? 1 : cps;
-    L->cl = cps >= kHidCluster ? kHidCluster : 1;
-    cps = cps / L->cl * L->cl;
-    L->cps = cps;
-    L->rpc = (d->N + cps - 1) / cps;
+    L->grid = hidden_grid(d);
+    const int cps = L->grid.cps;
     size_t off = 0;
     L->off_src = off;     off = align_up(off + (size_t)d->B * d->N * 4, 256);
     L->off_dst = off;     off = align_up(off + (size_t)d->B * d->N * 4, 256);
     L->off_wgt = off;     off = align_up(off + (size_t)d->B * d->n * 4, 256);
     L->off_meta = off;    off = align_up(off + (size_t)d->B * kMetaInts * 4, 256);
-    L->off_partial = off; off = align_up(off + (size_t)d->B * (cps / L->cl) * d->C * 4, 256);
+    L->off_partial = off; off = align_up(off + (size_t)d->B * (cps / L->grid.cl) * d->C * 4, 256);
     L->total = off;
     return true;
 }
 
 size_t merge_compact_workspace(const lvlm_dims* d) {
+    if (d && d->merge_mode == LVLM_W_NEAREST_KEPT) return nearest_kept_workspace(d);
     MergeLayout L;
     return merge_layout(d, &L) ? L.total : 0;
 }
@@ -201,7 +212,7 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
                      int64_t hid_stride_b, int64_t out_stride_b,   // in uint4
                      int V, int N, int i0, int n, int k, int rpc, int cl,
                      const int32_t* __restrict__ dst_map, const float* __restrict__ wgt,
-                     int32_t* meta, float* partial) {
+                     int32_t* meta, float* partial, uint4* __restrict__ scratch, int64_t scr_stride_b) {
     extern __shared__ __align__(16) float s_sum[];           // [V][8] this CTA's sums
     __shared__ int s_last;
     pdl_enter();
@@ -209,7 +220,8 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
     const uint4* hin = hidden + (int64_t)b * hid_stride_b;
     uint4* hout = out + (int64_t)b * out_stride_b;
     const int32_t* dst = dst_map + (int64_t)b * N;
-    const float* w = wgt + (int64_t)b * n - i0;               // indexed by sequence position
+    const float* w = wgt ? wgt + (int64_t)b * n - i0 : nullptr;   // indexed by sequence position
+    uint4* scr = scratch ? scratch + (int64_t)b * scr_stride_b : nullptr;
     const int i_lo = min(N, cta * rpc), i_hi = min(N, i_lo + rpc);
 
     float acc[CH][8];
@@ -225,8 +237,8 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int i = ib + u;
-            d[u] = i < i_hi ? dst[i] : -2;
-            wj[u] = (i < i_hi && i >= i0 && i < i0 + n) ? w[i] : 0.f;
+            d[u] = i < i_hi ? dst[i] : kNoRow;
+            wj[u] = (w && i < i_hi && i >= i0 && i < i0 + n) ? w[i] : 0.f;
 #pragma unroll
             for (int ci = 0; ci < CH; ++ci) {
                 const int c = tid + ci * kHidThreads;
@@ -241,6 +253,14 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
                     const int c = tid + ci * kHidThreads;
                     if (c < V) hout[(int64_t)d[u] * V + c] = x[u][ci];
                 }
+            } else if (d[u] <= -2 && d[u] != kNoRow) {        // a row set aside: scratch row -d-2
+                if (scr) {
+#pragma unroll
+                    for (int ci = 0; ci < CH; ++ci) {
+                        const int c = tid + ci * kHidThreads;
+                        if (c < V) scr[(int64_t)(-d[u] - 2) * V + c] = x[u][ci];
+                    }
+                }
             } else if (d[u] == -1) {
 #pragma unroll
                 for (int ci = 0; ci < CH; ++ci) {
@@ -253,6 +273,7 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
         }
     }
 
+    if (!w) return;                                           // no merged row in this mode
     // ---- clusters that touch the image span contribute a partial sum ---------------------------------
     const int rows_per_cluster = rpc * cl;
     const int cluster = cta / cl;
@@ -332,15 +353,31 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
 
 template <int CH>
 static lvlm_status launch_hidden_stream(const void* hidden, void* hidden_out, int64_t hid_sb, int64_t out_sb,
-                                        const lvlm_dims* d, const MergeLayout& L, const int32_t* dst_map,
-                                        const float* wgt, int32_t* meta, float* partial, cudaStream_t stream) {
+                                        const lvlm_dims* d, const HiddenGrid& L, const int32_t* dst_map,
+                                        const float* wgt, int32_t* meta, float* partial, void* scratch,
+                                        int64_t scr_sb, cudaStream_t stream) {
     const size_t smem = (size_t)L.V * 32;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(hidden_stream_kernel<CH>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     return launch_kernel(hidden_stream_kernel<CH>, dim3((unsigned)L.cps, (unsigned)d->B), dim3(kHidThreads), smem,
                          stream, L.cl, static_cast<const uint4*>(hidden), static_cast<uint4*>(hidden_out),
                          hid_sb / 8, out_sb / 8, L.V, d->N, d->i0, d->n, d->k, L.rpc, L.cl, dst_map, wgt, meta,
-                         partial);
+                         partial, static_cast<uint4*>(scratch), scr_sb / 8);
+}
+
+lvlm_status launch_hidden_rows(const void* hidden, void* hidden_out, int64_t hid_sb, int64_t out_sb,
+                               const lvlm_dims* d, const HiddenGrid& L, const int32_t* dst_map,
+                               const float* wgt, int32_t* meta, float* partial, void* scratch,
+                               int64_t scr_sb, cudaStream_t stream) {
+    const int chunks = (L.V + kHidThreads - 1) / kHidThreads;
+    if (chunks > kHidMaxChunks) return LVLM_ERR_UNSUPPORTED;  // more than 8192 channels
+    switch (chunks) {
+        case 1: return launch_hidden_stream<1>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
+        case 2: return launch_hidden_stream<2>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
+        case 3: return launch_hidden_stream<3>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
+        case 4: return launch_hidden_stream<4>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
+    }
+    return LVLM_ERR_UNSUPPORTED;
 }
 
 }  // namespace lvlm
@@ -359,10 +396,13 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     if ((Kc == nullptr) != (Vc == nullptr)) return LVLM_ERR_INVALID_ARG;
     if ((int)mode < 0 || (int)mode > LVLM_W_NEAREST_KEPT) return LVLM_ERR_INVALID_ARG;
     if (mode == LVLM_W_CUSTOM && !w_custom) return LVLM_ERR_INVALID_ARG;
-    if (mode == LVLM_W_NEAREST_KEPT) return LVLM_ERR_UNSUPPORTED;
     if (Kc) {
         if (d->Hkv <= 0 || d->cap < d->N) return LVLM_ERR_INVALID_ARG;
         if (d->D != kHeadDim) return LVLM_ERR_UNSUPPORTED;
+    }
+    if (mode == LVLM_W_NEAREST_KEPT) {    // no P_new row: N - (n - k) rows come out
+        L.r = d->n - d->k;
+        L.Nout = d->N - L.r;
     }
     const int64_t hid_sb = d->hid_stride_b ? d->hid_stride_b : (int64_t)d->N * d->C;
     const int64_t out_sb = hidden_out ? (d->out_stride_b ? d->out_stride_b : (int64_t)L.Nout * d->C) : hid_sb;
@@ -383,6 +423,9 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
                                           new_len, d->B, d->N);
         return LVLM_OK;
     }
+    if (mode == LVLM_W_NEAREST_KEPT)
+        return launch_nearest_kept(hidden, hidden_out, Kc, Vc, pos_ids, rank, d, mass, new_len, ws, ws_bytes,
+                                   dev_status, stream);
     if (!ws || !aligned256(ws) || ws_bytes < L.total) return LVLM_ERR_WORKSPACE;
     char* wsb = static_cast<char*>(ws);
     int32_t* src_map = reinterpret_cast<int32_t*>(wsb + L.off_src);
@@ -403,16 +446,8 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     }
 
     if (hidden_out) {
-        lvlm_status st;
-        const int chunks = (L.V + kHidThreads - 1) / kHidThreads;
-        if (chunks > kHidMaxChunks) return LVLM_ERR_UNSUPPORTED;       // more than 8192 channels
-        switch (chunks) {
-            case 1: st = launch_hidden_stream<1>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
-            case 2: st = launch_hidden_stream<2>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
-            case 3: st = launch_hidden_stream<3>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
-            case 4: st = launch_hidden_stream<4>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, stream); break;
-            default: return LVLM_ERR_UNSUPPORTED;
-        }
+        const lvlm_status st = launch_hidden_rows(hidden, hidden_out, hid_sb, out_sb, d, L.grid, dst_map, wgt, meta,
+                                                  partial, nullptr, 0, stream);
         if (st != LVLM_OK) return st;
     } else {
         lvlm_status st = launch_inplace_compact(hidden, nullptr, hid_sb * 2, 0, d->B, 1, L.V,

@@ -347,3 +347,66 @@ def test_cfg1_pipeline():
     out = L.decode_attn(qd.cuda(), Kd, Vd, ld, acc_score=ad)
     assert_rows_close(f64(out), o_dec["out"], what="cfg1 decode")
     assert_scores_close(ad.cpu().numpy()[:, :, :m], o_dec["acc_score"][:, :, :m], what="cfg1 acc")
+
+
+# ------------------------------------------------------------------ nearest-kept merge (spec variant)
+NK_CASES = [  # B, N, i0, n, C, k, Hkv, with_mass, with_kv
+    (1, 40, 3, 30, 64, 7, 1, False, False), (2, 700, 5, 640, 256, 300, 2, True, True),
+    (1, 1500, 0, 1400, 200, 130, 2, False, True), (3, 333, 2, 300, 1024, 299, 1, True, False),
+    (1, 520, 8, 500, 3584, 1, 4, True, True), (2, 600, 0, 600, 512, 600, 2, False, True),
+]
+
+
+@pytest.mark.parametrize("case", NK_CASES)
+def test_merge_nearest_kept(case):
+    B, N, i0, n, C, k, Hkv, with_mass, with_kv = case
+    r = np.random.default_rng(N + C)
+    # clustered rows so that similarities are well separated, plus noise
+    cent = r.normal(size=(24, C))
+    hidden = cent[r.integers(0, 24, size=(B, N))] + 0.4 * r.normal(size=(B, N, C))
+    hidden = torch.from_numpy(hidden.astype(np.float32)).to(torch.bfloat16)
+    score = r.random((B, n)).astype(np.float32)
+    rank, _, _, _ = O.select_topk(score, k)
+    pos = np.tile(np.arange(N, dtype=np.int32) * 3, (B, 1))
+    mass = (1 + r.integers(0, 4, size=(B, N))).astype(np.float32) if with_mass else None
+    Kc = torch.from_numpy(r.normal(size=(B, Hkv, N, 128)).astype(np.float32)).to(torch.bfloat16) if with_kv else None
+    Vc = torch.from_numpy(r.normal(size=(B, Hkv, N, 128)).astype(np.float32)).to(torch.bfloat16) if with_kv else None
+    ref = O.nearest_kept_merge(f64(hidden), rank, i0, n, k, mass=mass)
+
+    hd, rd = hidden.cuda(), torch.from_numpy(rank).cuda()
+    Kd, Vd = (Kc.cuda(), Vc.cuda()) if with_kv else (None, None)
+    pd = torch.from_numpy(pos).cuda()
+    md = torch.from_numpy(mass).cuda() if with_mass else None
+    d = L.merge_dims(hd, rd, i0=i0, k=k, Kc=Kd)
+    d.merge_mode = L.W_NEAREST_KEPT
+    ws = L.alloc_workspace(L.OP_MERGE_COMPACT, d, hd.device)
+    flag = status_tensor()
+    out, new_len = L.merge_compact(hd, rd, i0=i0, k=k, mode=L.W_NEAREST_KEPT, Kc=Kd, Vc=Vd, pos_ids=pd, mass=md,
+                                   ws=ws, dev_status=flag)
+    torch.cuda.synchronize()
+    rr = n - k
+    assert flag.item() == 0 and out.shape == (B, N - rr, C) and (i32(new_len) == N - rr).all()
+    if rr == 0:
+        assert torch.equal(out, hd)
+        return
+    g_assign = i32(L.nearest_assignment(ws, B, rr))
+    # a different choice must be a near-tie of the two similarities in the oracle
+    for b, q in zip(*np.nonzero(g_assign != ref["assign"])):
+        x = f64(hidden)[b, i0:i0 + n]
+        kept = np.nonzero(rank[b] < k)[0]
+        dtok = np.nonzero(rank[b] >= k)[0][q]
+        cos = lambda t: float(x[kept[t]] @ x[dtok] / np.linalg.norm(x[kept[t]]) / np.linalg.norm(x[dtok]))
+        a, c = cos(ref["assign"][b, q]), cos(g_assign[b, q])
+        assert abs(a - c) <= 1e-4 * max(abs(a), abs(c)), "assignment differs and is not a near-tie"
+    want = O.nearest_kept_merge(f64(hidden), rank, i0, n, k, mass=mass, Kc=f64(Kc) if with_kv else None,
+                                Vc=f64(Vc) if with_kv else None, pos_ids=pos, assign=g_assign)
+    M = N - rr
+    assert_rows_close(f64(out), want["hidden"], what="merged hidden rows")
+    assert torch.equal(out[:, :i0], hd[:, :i0]) and torch.equal(out[:, i0 + k:], hd[:, i0 + n:])
+    assert np.array_equal(i32(pd)[:, :M], want["pos_ids"])
+    if with_mass:
+        assert np.array_equal(md.cpu().numpy()[:, :M], want["mass"])
+    if with_kv:
+        assert_rows_close(f64(Kd)[:, :, :M], want["Kc"], what="merged K rows")
+        assert_rows_close(f64(Vd)[:, :, :M], want["Vc"], what="merged V rows")
+        assert np.array_equal(f64(Kd)[:, :, i0 + k:M], f64(Kc)[:, :, i0 + n:])       # text rows only move
