@@ -22,7 +22,10 @@ class ReduceStage:
 
     def __init__(self, B, N, C, H, Hkv, cap, i0, n, M, device, want_head=False, mode=L.W_LINEAR_RANK):
         self.B, self.N, self.C, self.H, self.Hkv, self.cap = B, N, C, H, Hkv, cap
-        self.i0, self.n, self.M, self.k, self.mode = i0, n, M, M - 1, mode
+        # M image tokens come out: with a merged token P_new, k = M - 1 tokens stay intact; in the
+        # nearest-kept mode there is no extra token and k = M
+        self.i0, self.n, self.M, self.mode = i0, n, M, mode
+        self.k = M if mode == L.W_NEAREST_KEPT else M - 1
         self.q_lo, self.q_hi = i0 + n, N
         self.Nout = L.merged_rows(N, n, self.k, mode)
         f32, i32 = torch.float32, torch.int32
@@ -34,7 +37,7 @@ class ReduceStage:
         self.status = torch.zeros(1, dtype=i32, device=device)
         ds = L.Dims(B=B, H=H, Hkv=Hkv, D=128, N=N, cap=cap, i0=i0, n=n, q_lo=self.q_lo,
                     q_hi=self.q_hi, causal=1)
-        dm = L.Dims(B=B, N=N, C=C, Hkv=Hkv, D=128, cap=cap, i0=i0, n=n, k=self.k)
+        dm = L.Dims(B=B, N=N, C=C, Hkv=Hkv, D=128, cap=cap, i0=i0, n=n, k=self.k, merge_mode=int(mode))
         self.ws_score = L.alloc_workspace(L.OP_SCORE_TOKENS, ds, device)
         self.ws_merge = L.alloc_workspace(L.OP_MERGE_COMPACT, dm, device)
 
@@ -64,6 +67,10 @@ class ReduceStage:
 
     def bytes_merge_kv(self):
         return self.B * self.Hkv * (self.N + self.Nout) * 128 * 2 * 2
+
+    def flops_similarity(self):
+        """Nearest-kept mode: dropped x kept similarity, 2 r k C per sequence."""
+        return 2.0 * (self.n - self.k) * self.k * self.C * self.B
 
     def flops_score(self):
         # text window rows x visible keys x D x heads, two passes (normaliser, column sums)

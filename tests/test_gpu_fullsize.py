@@ -198,3 +198,31 @@ def test_cfg2_beta_compression_then_decode_full_size():
             assert np.array_equal(f64(dec.V[i])[0, g, :m], od["Vc"][0, g, :m].astype(np.float64))
             assert_scores_close(dec.acc[i].cpu().numpy()[0, g, :m], od["acc_score"][0, g, :m], what="acc_score")
         assert_rows_close(f64(dec.out[i]), od["out"], what="decode output over the ragged cache")
+
+
+@pytest.mark.parametrize("wname,b", [("cfg2", 0), ("cfg3", 5)])
+def test_nearest_kept_stage_full_size(wname, b):
+    """First reduction stage of a workload in the nearest-kept merge mode, one sequence checked."""
+    w, dev = I.WORKLOADS[wname], torch.device("cuda", 0)
+    layer, M = w.stages[0]
+    st = P.ReduceStage(w.B, w.N, w.C, w.H, w.Hkv, w.N, w.i0, w.n, M, dev, mode=L.W_NEAREST_KEPT)
+    hidden = I.hidden_states(w, dev)
+    pos = torch.arange(w.N, dtype=torch.int32, device=dev)[None].repeat(w.B, 1).contiguous()
+    q, K, V = I.layer_qkv(w, layer, pos, dev)
+    K0, V0 = K.clone(), V.clone()
+    out = st.run(hidden, q[:, st.q_lo:st.q_hi].contiguous(), K, V, pos)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0 and np.all(i32(st.new_len) == st.Nout) and st.Nout == w.N - (w.n - M)
+    rr = w.n - M
+    g_rank = i32(st.rank)[b:b + 1]
+    g_assign = i32(L.nearest_assignment(st.ws_merge, w.B, rr))[b:b + 1]
+    ref = O.nearest_kept_merge(f64(hidden[b:b + 1]), g_rank, w.i0, w.n, M)
+    diff = np.nonzero(g_assign[0] != ref["assign"][0])[0]
+    for qd in diff:       # the GPU's choice is the oracle's runner-up, within the near-tie bound
+        a, c = ref["sim_best"][0, qd], ref["sim_second"][0, qd]
+        assert abs(a - c) <= 1e-4 * max(abs(a), abs(c)), "assignment differs and is not a near-tie"
+    want = O.nearest_kept_merge(f64(hidden[b:b + 1]), g_rank, w.i0, w.n, M, Kc=f64(K0[b:b + 1]),
+                                Vc=f64(V0[b:b + 1]), assign=g_assign)
+    assert_rows_close(f64(out[b]), want["hidden"][0], what="merged hidden rows")
+    assert_rows_close(f64(K[b, :, :st.Nout]), want["Kc"][0], what="merged K rows")
+    assert_rows_close(f64(V[b, :, :st.Nout]), want["Vc"][0], what="merged V rows")
