@@ -1,67 +1,122 @@
 // lvlm_select_topk: total order of the image tokens by (score descending, index ascending).
 // Section 3.2.1, paragraph 4: the tokens with the highest scores form P_unmerged, the others
 // form P_merged, "reordered by their importance".
+//
+// The rank of a token is the number of tokens that come before it in that order, so it can be
+// counted directly: nothing iterative, every token independent of the others.  Keys are 64-bit
+// (order-preserving image of the score << 32 | index), so the order is total and ties go to the
+// lower index.  grid (blocks of 256 tokens, S, B): a CTA counts, for its 256 tokens, the keys of
+// one slice of the sequence that are smaller (shared memory, every thread reads the same key at
+// the same time); the S CTAs of a cluster add their counts through distributed shared memory.
+// The optional outputs (kept list, near-tie count) come from a second, small kernel.
 #include "common.cuh"
-#include "sort.cuh"
 
 namespace lvlm {
 
-// One CTA per sequence.  Shared memory: P 64-bit keys (score key << 32 | index) followed by
-// n int32 ranks.  The stable order falls out of the index in the low word.
-__global__ void __launch_bounds__(1024)
-select_rank_kernel(const float* __restrict__ score, int64_t stride, int n, int k, int P,
-                   int32_t* __restrict__ rank, int32_t* __restrict__ kept_idx,
-                   int32_t* __restrict__ near_tie, int32_t* dev_status) {
+constexpr int kSelThreads = 256;
+constexpr int kSelMaxCluster = 8;
+
+__device__ __forceinline__ uint32_t sel_cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void sel_cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ int sel_ld_cluster(const int* my_smem, uint32_t rank) {
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    int v;
+    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+// Clusters of S CTAs along y.  slice_len is even; the slice is padded with keys that are larger
+// than every real key.
+__global__ void __launch_bounds__(kSelThreads)
+select_count_kernel(const float* __restrict__ score, int64_t stride, int n, int S, int slice_len,
+                    int32_t* __restrict__ rank, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* keys = reinterpret_cast<uint64_t*>(smem_raw);
-    int32_t* srank = reinterpret_cast<int32_t*>(keys + P);
+    uint64_t* sk = reinterpret_cast<uint64_t*>(smem_raw);            // [slice_len]
+    __shared__ int s_cnt[kSelThreads];
+    pdl_enter();
+    const int b = blockIdx.z, s = (int)sel_cluster_rank(), tid = threadIdx.x;
+    const float* row = score + (int64_t)b * stride;
+    const int i_lo = s * slice_len;
+    bool nonfinite = false, ignored = false;
+    for (int i = tid; i < slice_len; i += kSelThreads) {
+        const int gi = i_lo + i;
+        sk[i] = gi < n ? (((uint64_t)desc_key(row[gi], &ignored) << 32) | (uint32_t)gi) : ~0ull;
+    }
+    const int j = blockIdx.x * kSelThreads + tid;
+    const uint64_t kj = j < n ? (((uint64_t)desc_key(row[j], &nonfinite) << 32) | (uint32_t)j) : 0ull;
+    if (nonfinite && s == 0 && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
+    __syncthreads();
+    int cnt = 0;
+    const ulonglong2* sk2 = reinterpret_cast<const ulonglong2*>(sk);
+#pragma unroll 4
+    for (int i = 0; i < slice_len / 2; ++i) {
+        const ulonglong2 v = sk2[i];
+        cnt += (v.x < kj) + (v.y < kj);
+    }
+    if (S == 1) {
+        if (j < n) rank[(int64_t)b * n + j] = cnt;
+        return;
+    }
+    s_cnt[tid] = cnt;
+    sel_cluster_barrier();
+    if (s == 0 && j < n) {
+        int tot = 0;
+        for (int r = 0; r < S; ++r) tot += sel_ld_cluster(&s_cnt[tid], r);
+        rank[(int64_t)b * n + j] = tot;
+    }
+    sel_cluster_barrier();                                            // nobody leaves while its counts are read
+}
+
+// One CTA per sequence: the kept tokens in ascending order (prefix sum of rank < k over the index) and
+// the number of near-ties among neighbours (p, p+1) of the order with p+1 >= k.
+__global__ void __launch_bounds__(1024)
+select_aux_kernel(const float* __restrict__ score, int64_t stride, int n, int k,
+                  const int32_t* __restrict__ rank, int32_t* __restrict__ kept_idx,
+                  int32_t* __restrict__ near_tie) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    int32_t* order = reinterpret_cast<int32_t*>(smem_raw);           // [n] token at every place of the order
     __shared__ int scan_scratch[33];
     __shared__ int s_near;
-
     pdl_enter();
     const int b = blockIdx.x;
     const float* row = score + (int64_t)b * stride;
-    bool nonfinite = false;
+    const int32_t* rk = rank + (int64_t)b * n;
     if (threadIdx.x == 0) s_near = 0;
-    for (int j = threadIdx.x; j < P; j += blockDim.x) {
-        uint64_t key = ~0ull;
-        if (j < n) key = ((uint64_t)desc_key(row[j], &nonfinite) << 32) | (uint32_t)j;
-        keys[j] = key;
+    for (int j = threadIdx.x; j < n; j += blockDim.x) {
+        const int p = rk[j];
+        if (p >= 0 && p < n) order[p] = j;
     }
-    if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
     __syncthreads();
-    block_bitonic_sort(keys, P);
-
-    int near = 0;
-    for (int p = threadIdx.x; p < n; p += blockDim.x) {
-        const int idx = (int)(uint32_t)keys[p];
-        srank[idx] = p;
-        rank[(int64_t)b * n + idx] = p;
-        if (near_tie && p + 1 >= k && p + 1 < n) {
-            const float a = row[idx];
-            const float c = row[(int)(uint32_t)keys[p + 1]];
+    if (near_tie) {
+        int near = 0;
+        for (int p = threadIdx.x + max(k - 1, 0); p + 1 < n; p += blockDim.x) {
+            const float a = row[order[p]], c = row[order[p + 1]];
             const float dgap = __fsub_rn(a, c);
             const float t = __fmul_rn(1e-4f, fabsf(a));
             if (dgap < t) ++near;
         }
-    }
-    if (near_tie) {
         near = warp_sum(near);
         if ((threadIdx.x & 31) == 0 && near) atomicAdd(&s_near, near);
+        __syncthreads();
+        if (threadIdx.x == 0) near_tie[b] = s_near;
     }
-    __syncthreads();
-    if (near_tie && threadIdx.x == 0) near_tie[b] = s_near;
-
     if (kept_idx && k > 0) {
-        // kept tokens in ascending index order: prefix sum of (rank < k) over the index
         const int per = (n + blockDim.x - 1) / blockDim.x;
         const int j0 = min(n, (int)threadIdx.x * per), j1 = min(n, j0 + per);
         int cnt = 0;
-        for (int j = j0; j < j1; ++j) cnt += srank[j] < k;
+        for (int j = j0; j < j1; ++j) cnt += rk[j] < k;
         int total;
         int off = block_exclusive_scan(cnt, scan_scratch, &total);
         for (int j = j0; j < j1; ++j)
-            if (srank[j] < k) kept_idx[(int64_t)b * k + off++] = j;
+            if (rk[j] < k && off < k) kept_idx[(int64_t)b * k + off++] = j;
     }
 }
 
@@ -70,19 +125,49 @@ select_rank_kernel(const float* __restrict__ score, int64_t stride, int n, int k
 extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_stride,
                                          int k, int32_t* rank, int32_t* kept_idx,
                                          int32_t* near_tie, void* ws, size_t ws_bytes,
-                                         int32_t* dev_status, void* stream) {
+                                         int32_t* dev_status, void* stream_) {
     using namespace lvlm;
     (void)ws; (void)ws_bytes;
+    cudaStream_t stream = (cudaStream_t)stream_;
     if (!score || !rank || B <= 0 || n <= 0 || k < 0 || k > n) return LVLM_ERR_INVALID_ARG;
     if (score_stride == 0) score_stride = n;
     if (score_stride < n) return LVLM_ERR_INVALID_ARG;
     if (n > kMaxSortN) return LVLM_ERR_UNSUPPORTED;
-    const int P = next_pow2(n < 2 ? 2 : n);
-    int threads = P / 2;
-    threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
-    const size_t smem = (size_t)P * 8 + (size_t)n * 4;
-    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_rank_kernel,
+    const int jblocks = (n + kSelThreads - 1) / kSelThreads;
+    // slices: up to eight CTAs of 256 threads per SM, at least 256 keys per slice
+    int S = 1;
+    while (S < kSelMaxCluster && (int64_t)jblocks * B * (2 * S) <= 8 * 148 && n / (2 * S) >= 256) S *= 2;
+    int slice_len = (n + S - 1) / S;
+    slice_len = (slice_len + 1) & ~1;
+    const size_t smem = (size_t)slice_len * 8;
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_count_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    return launch_kernel(select_rank_kernel, dim3(B), dim3(threads), smem, (cudaStream_t)stream, 1,
-                         score, score_stride, n, k, P, rank, kept_idx, near_tie, dev_status);
+    // clusters along y need a launch of their own shape: grid (jblocks, S, B), cluster (1, S, 1)
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(jblocks, S, B);
+        cfg.blockDim = dim3(kSelThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[2];
+        int na = 0;
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = (unsigned)S; attr[na].val.clusterDim.z = 1;
+        ++na;
+        if (pdl_enabled()) {
+            attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[na].val.programmaticStreamSerializationAllowed = 1;
+            ++na;
+        }
+        cfg.attrs = attr;
+        cfg.numAttrs = na;
+        LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, select_count_kernel, score, score_stride, n, S, slice_len,
+                                               rank, dev_status));
+    }
+    if (!kept_idx && !near_tie) return LVLM_OK;
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_aux_kernel,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+    const int threads = n >= 1024 ? 1024 : ((n + 31) / 32) * 32;
+    return launch_kernel(select_aux_kernel, dim3(B), dim3(threads), (size_t)n * 4, stream, 1,
+                         score, score_stride, n, k, rank, kept_idx, near_tie);
 }
