@@ -201,9 +201,9 @@ __device__ __forceinline__ float4 hid_ld_cluster_f4(const float* my_smem, uint32
 }
 
 // Hidden states, out of place.  grid (CTAs per sequence, B), clusters of `cl` CTAs along x.  A CTA
-// owns `rpc` consecutive INPUT rows and reads each of them exactly once, four rows in flight: a kept
+// takes every grid.x-th group of four consecutive INPUT rows and reads each row exactly once: a kept
 // row goes to its destination, a merged row is added, times its weight, to fp32 sums the thread
-// keeps for its columns (rows in increasing order).  The CTAs of a cluster add their sums in rank
+// keeps for its columns (its rows in increasing order).  The CTAs of a cluster add their sums in rank
 // order through distributed shared memory and park one partial per cluster; the last cluster of
 // the sequence to finish adds the partials in cluster order, rounds once to bf16 and writes P_new.
 template <int CH>
@@ -222,7 +222,8 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
     const int32_t* dst = dst_map + (int64_t)b * N;
     const float* w = wgt ? wgt + (int64_t)b * n - i0 : nullptr;   // indexed by sequence position
     uint4* scr = scratch ? scratch + (int64_t)b * scr_stride_b : nullptr;
-    const int i_lo = min(N, cta * rpc), i_hi = min(N, i_lo + rpc);
+    const int i_hi = N;
+    (void)rpc;
 
     float acc[CH][8];
 #pragma unroll
@@ -230,7 +231,9 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
 
-    for (int ib = i_lo; ib < i_hi; ib += 4) {
+    // groups of four rows are dealt out round robin, so that every CTA gets the same mix of kept
+    // rows (read and written) and merged rows (read only)
+    for (int ib = cta * 4; ib < i_hi; ib += (int)gridDim.x * 4) {
         int d[4];
         float wj[4];
         uint4 x[4][CH];
@@ -275,10 +278,8 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
 
     if (!w) return;                                           // no merged row in this mode
     // ---- clusters that touch the image span contribute a partial sum ---------------------------------
-    const int rows_per_cluster = rpc * cl;
     const int cluster = cta / cl;
-    const int q_first = i0 / rows_per_cluster, q_last = (i0 + n - 1) / rows_per_cluster;
-    if (cluster < q_first || cluster > q_last) return;        // the whole cluster leaves together
+    const int q_first = 0, q_last = (int)gridDim.x / cl - 1;  // every cluster has seen merged rows
     const int rank = (int)hid_cluster_rank();
 #pragma unroll
     for (int ci = 0; ci < CH; ++ci) {
