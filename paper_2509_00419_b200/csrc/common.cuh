@@ -44,11 +44,11 @@ __device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_launch_dependents(
 
 bool pdl_enabled();            // lvlm.cu; test hook lvlm_debug_set_pdl switches it off
 
-// Launches `kernel` with programmatic stream serialisation and, when cluster_x > 1, clusters of
-// cluster_x CTAs along x.
+// Launches `kernel` with programmatic stream serialisation and thread-block clusters of the given shape
+// (1, 1, 1 = no clusters).
 template <typename... KArgs, typename... Args>
-inline lvlm_status launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                 cudaStream_t stream, int cluster_x, Args... args) {
+inline lvlm_status launch_kernel_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                         cudaStream_t stream, dim3 cluster, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -56,11 +56,11 @@ inline lvlm_status launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     int na = 0;
-    if (cluster_x > 1) {
+    if (cluster.x * cluster.y * cluster.z > 1) {
         attr[na].id = cudaLaunchAttributeClusterDimension;
-        attr[na].val.clusterDim.x = (unsigned)cluster_x;
-        attr[na].val.clusterDim.y = 1;
-        attr[na].val.clusterDim.z = 1;
+        attr[na].val.clusterDim.x = cluster.x;
+        attr[na].val.clusterDim.y = cluster.y;
+        attr[na].val.clusterDim.z = cluster.z;
         ++na;
     }
     if (pdl_enabled()) {
@@ -71,6 +71,14 @@ inline lvlm_status launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     cfg.attrs = attr;
     cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess ? LVLM_OK : LVLM_ERR_CUDA;
+}
+
+// The same with clusters of cluster_x CTAs along x.
+template <typename... KArgs, typename... Args>
+inline lvlm_status launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, int cluster_x, Args... args) {
+    return launch_kernel_cluster(kernel, grid, block, smem, stream, dim3(cluster_x < 1 ? 1 : cluster_x, 1, 1),
+                                 args...);
 }
 
 // ---- bf16 <-> fp32 on packed words -------------------------------------------------

@@ -23,11 +23,13 @@ constexpr int kHidMaxChunks = 4;       // column groups per thread: rows up to 4
 constexpr int kNoRow = -2147483647 - 1;  // marks a slot of the four-row group that lies past the CTA's rows
 constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
 
-// One wave of four CTAs per SM over the whole batch, at least 8 input rows each; clusters of 8.
+// One wave of CTAs over the whole batch (four per SM fit for rows up to 4096 channels, two beyond:
+// the registers of the row groups in flight decide), at least 8 input rows each; clusters of 8.
 HiddenGrid hidden_grid(const lvlm_dims* d) {
     HiddenGrid g;
     g.V = d->C / 8;
-    int cps = (4 * 148) / d->B;
+    const int per_sm = (g.V + kHidThreads - 1) / kHidThreads <= 2 ? 4 : 2;
+    int cps = (per_sm * 148) / d->B;
     const int max_by_rows = (d->N + 7) / 8;
     cps = cps > max_by_rows ? max_by_rows : cps;
     cps = cps < 1 ? 1 : cps;

@@ -11,7 +11,7 @@
 //   sim       dropped x kept similarity on the tensor cores (tcgen05, accumulators in TMEM, operands by
 //             TMA), arg-max per dropped row in the epilogue, merged over column splits with atomicMax
 //             on (similarity, ~index) keys
-//   group     one CTA per sequence: dropped tokens sorted by (kept token, own index) -> segments
+//   group     dropped tokens sorted by (kept token, own index) by rank counting -> segments
 //   merge     every kept row becomes the mass-weighted mean of itself and its segment, in token order
 //   K, V      the same mean per KV head into scratch, text rows shifted down in place, means stored
 //   mass      token masses compacted in place
@@ -19,7 +19,7 @@
 #include "compact.cuh"
 #include "merge.cuh"
 #include "sm100.cuh"
-#include "sort.cuh"
+#include "rank_count.cuh"
 
 namespace lvlm {
 
@@ -28,7 +28,7 @@ using namespace sm100;
 struct NkLayout {
     int r, Nout, V;
     HiddenGrid grid;
-    size_t off_assign, off_src, off_dst, off_kept, off_drop, off_inv, off_best, off_order, off_seg,
+    size_t off_assign, off_src, off_dst, off_kept, off_drop, off_inv, off_best, off_order, off_sorted, off_seg,
            off_meta, off_newmass, off_scratch, off_kvtmp, total;
 };
 
@@ -50,6 +50,7 @@ static bool nk_layout(const lvlm_dims* d, NkLayout* L) {
     L->off_inv = off;     off = align_up(off + B * (k ? k : 1) * 4, 256);
     L->off_best = off;    off = align_up(off + B * (r ? r : 1) * 8, 256);
     L->off_order = off;   off = align_up(off + B * (r ? r : 1) * 4, 256);
+    L->off_sorted = off;  off = align_up(off + B * (r ? r : 1) * 4, 256);
     L->off_seg = off;     off = align_up(off + B * (k + 1) * 4, 256);
     L->off_meta = off;    off = align_up(off + B * kMetaInts * 4, 256);
     L->off_newmass = off; off = align_up(off + B * (k ? k : 1) * 4, 256);
@@ -152,36 +153,44 @@ nk_norm_kernel(const uint4* __restrict__ out, int64_t out_stride_b, int V, int i
 }
 
 // ---- group -----------------------------------------------------------------------------------------
-// One CTA per sequence: decodes the winning kept token of every dropped token, sorts the dropped
-// tokens by (kept token, own order) and finds where every kept token's segment starts.
-__global__ void __launch_bounds__(1024)
-nk_group_kernel(const unsigned long long* __restrict__ best, int r, int k, int P,
-                int32_t* __restrict__ assign, int32_t* __restrict__ order, int32_t* __restrict__ seg) {
+// Dropped tokens sorted by (kept token they go to, own order), by counting ranks: grid (blocks of 256
+// dropped tokens, S, B), clusters (1, S, 1).  Writes the assignment, the sorted order and the kept
+// token at every place of that order; a second kernel finds where every kept token's segment starts.
+__global__ void __launch_bounds__(kRankThreads)
+nk_group_kernel(const unsigned long long* __restrict__ best, int r, int k, int S, int slice_len,
+                int32_t* __restrict__ assign, int32_t* __restrict__ order, int32_t* __restrict__ sorted_t) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* keys = reinterpret_cast<uint64_t*>(smem_raw);
+    __shared__ int s_cnt[kRankThreads];
     pdl_enter();
-    const int b = blockIdx.x;
-    for (int q = threadIdx.x; q < P; q += blockDim.x) {
-        uint64_t key = ~0ull;
-        if (q < r) {
-            const uint32_t t = 0xFFFFFFFFu - (uint32_t)(best[(int64_t)b * r + q] & 0xFFFFFFFFull);
-            const uint32_t tt = t < (uint32_t)k ? t : 0u;           // nothing won (k == 0 cannot happen here)
-            assign[(int64_t)b * r + q] = (int)tt;
-            key = ((uint64_t)tt << 32) | (uint32_t)q;
-        }
-        keys[q] = key;
+    const int b = blockIdx.z;
+    const unsigned long long* bb = best + (int64_t)b * r;
+    auto key_of = [&](int q) {
+        const uint32_t t = 0xFFFFFFFFu - (uint32_t)(bb[q] & 0xFFFFFFFFull);
+        return ((uint64_t)(t < (uint32_t)k ? t : 0u) << 32) | (uint32_t)q;     // nothing won: kept token 0
+    };
+    int p = 0;
+    if (rank_by_counting(key_of, r, S, slice_len, reinterpret_cast<uint64_t*>(smem_raw), s_cnt, &p)) {
+        const int q = blockIdx.x * kRankThreads + threadIdx.x;
+        const int t = (int)(key_of(q) >> 32);
+        assign[(int64_t)b * r + q] = t;
+        order[(int64_t)b * r + p] = q;
+        sorted_t[(int64_t)b * r + p] = t;
     }
-    __syncthreads();
-    block_bitonic_sort(keys, P);
-    for (int p = threadIdx.x; p < r; p += blockDim.x) order[(int64_t)b * r + p] = (int)(uint32_t)keys[p];
-    for (int t = threadIdx.x; t <= k; t += blockDim.x) {            // first sorted position with kept token >= t
-        int lo = 0, hi = r;
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if ((uint32_t)(keys[mid] >> 32) < (uint32_t)t) lo = mid + 1; else hi = mid;
-        }
-        seg[(int64_t)b * (k + 1) + t] = lo;
+}
+
+// seg[t] = first place of the sorted order whose kept token is >= t (t = 0..k).
+__global__ void __launch_bounds__(256)
+nk_seg_kernel(const int32_t* __restrict__ sorted_t, int r, int k, int32_t* __restrict__ seg) {
+    pdl_enter();
+    const int b = blockIdx.y, t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t > k) return;
+    const int32_t* st = sorted_t + (int64_t)b * r;
+    int lo = 0, hi = r;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (st[mid] < t) lo = mid + 1; else hi = mid;
     }
+    seg[(int64_t)b * (k + 1) + t] = lo;
 }
 
 // ---- merge of the hidden rows ------------------------------------------------------------------------
@@ -532,7 +541,7 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
     NkLayout L;
     if (!nk_layout(d, &L) || d->k < 1) return LVLM_ERR_INVALID_ARG;
     if (!hidden_out || hidden_out == hidden) return LVLM_ERR_UNSUPPORTED;     // out of place only
-    if (L.r > kMaxSortN) return LVLM_ERR_UNSUPPORTED;
+    if (L.r > kMaxSortN) return LVLM_ERR_UNSUPPORTED;          // one slice of the keys has to fit in shared memory
     if (!ws || !aligned256(ws) || ws_bytes < L.total) return LVLM_ERR_WORKSPACE;
     const int64_t hid_sb = d->hid_stride_b ? d->hid_stride_b : (int64_t)d->N * d->C;
     const int64_t out_sb = d->out_stride_b ? d->out_stride_b : (int64_t)L.Nout * d->C;
@@ -548,6 +557,7 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
     float* inv_norm = reinterpret_cast<float*>(wsb + L.off_inv);
     unsigned long long* best = reinterpret_cast<unsigned long long*>(wsb + L.off_best);
     int32_t* order = reinterpret_cast<int32_t*>(wsb + L.off_order);
+    int32_t* sorted_t = reinterpret_cast<int32_t*>(wsb + L.off_sorted);
     int32_t* seg = reinterpret_cast<int32_t*>(wsb + L.off_seg);
     int32_t* meta = reinterpret_cast<int32_t*>(wsb + L.off_meta);
     float* newmass = reinterpret_cast<float*>(wsb + L.off_newmass);
@@ -592,13 +602,16 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
         if (st != LVLM_OK) return st;
     }
     {
-        const int P = next_pow2(L.r < 2 ? 2 : L.r);
-        int threads = P / 2;
-        threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
+        int S, slice_len;
+        rank_shape(L.r, d->B, &S, &slice_len);
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(nk_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  kMaxDynSmem));
-        st = launch_kernel(nk_group_kernel, dim3(d->B), dim3(threads), (size_t)P * 8, stream, 1,
-                           best, L.r, d->k, P, assign, order, seg);
+        st = launch_kernel_cluster(nk_group_kernel, dim3((L.r + kRankThreads - 1) / kRankThreads, S, d->B),
+                                   dim3(kRankThreads), (size_t)slice_len * 8, stream, dim3(1, S, 1),
+                                   best, L.r, d->k, S, slice_len, assign, order, sorted_t);
+        if (st != LVLM_OK) return st;
+        st = launch_kernel(nk_seg_kernel, dim3((d->k + 1 + 255) / 256, d->B), dim3(256), 0, stream, 1,
+                           sorted_t, L.r, d->k, seg);
         if (st != LVLM_OK) return st;
     }
     const int chunks = (L.V + kNkThreads - 1) / kNkThreads;

@@ -10,69 +10,26 @@
 // the same time); the S CTAs of a cluster add their counts through distributed shared memory.
 // The optional outputs (kept list, near-tie count) come from a second, small kernel.
 #include "common.cuh"
+#include "rank_count.cuh"
 
 namespace lvlm {
 
-constexpr int kSelThreads = 256;
-constexpr int kSelMaxCluster = 8;
-
-__device__ __forceinline__ uint32_t sel_cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void sel_cluster_barrier() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n"
-                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-}
-__device__ __forceinline__ int sel_ld_cluster(const int* my_smem, uint32_t rank) {
-    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
-    int v;
-    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
-    return v;
-}
-
-// Clusters of S CTAs along y.  slice_len is even; the slice is padded with keys that are larger
-// than every real key.
-__global__ void __launch_bounds__(kSelThreads)
+// grid (blocks of 256 tokens, S, B), clusters (1, S, 1).
+__global__ void __launch_bounds__(kRankThreads)
 select_count_kernel(const float* __restrict__ score, int64_t stride, int n, int S, int slice_len,
                     int32_t* __restrict__ rank, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* sk = reinterpret_cast<uint64_t*>(smem_raw);            // [slice_len]
-    __shared__ int s_cnt[kSelThreads];
+    __shared__ int s_cnt[kRankThreads];
     pdl_enter();
-    const int b = blockIdx.z, s = (int)sel_cluster_rank(), tid = threadIdx.x;
+    const int b = blockIdx.z;
     const float* row = score + (int64_t)b * stride;
-    const int i_lo = s * slice_len;
-    bool nonfinite = false, ignored = false;
-    for (int i = tid; i < slice_len; i += kSelThreads) {
-        const int gi = i_lo + i;
-        sk[i] = gi < n ? (((uint64_t)desc_key(row[gi], &ignored) << 32) | (uint32_t)gi) : ~0ull;
-    }
-    const int j = blockIdx.x * kSelThreads + tid;
-    const uint64_t kj = j < n ? (((uint64_t)desc_key(row[j], &nonfinite) << 32) | (uint32_t)j) : 0ull;
-    if (nonfinite && s == 0 && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
-    __syncthreads();
+    bool nonfinite = false;
+    auto key_of = [&](int i) { return ((uint64_t)desc_key(row[i], &nonfinite) << 32) | (uint32_t)i; };
     int cnt = 0;
-    const ulonglong2* sk2 = reinterpret_cast<const ulonglong2*>(sk);
-#pragma unroll 4
-    for (int i = 0; i < slice_len / 2; ++i) {
-        const ulonglong2 v = sk2[i];
-        cnt += (v.x < kj) + (v.y < kj);
-    }
-    if (S == 1) {
-        if (j < n) rank[(int64_t)b * n + j] = cnt;
-        return;
-    }
-    s_cnt[tid] = cnt;
-    sel_cluster_barrier();
-    if (s == 0 && j < n) {
-        int tot = 0;
-        for (int r = 0; r < S; ++r) tot += sel_ld_cluster(&s_cnt[tid], r);
-        rank[(int64_t)b * n + j] = tot;
-    }
-    sel_cluster_barrier();                                            // nobody leaves while its counts are read
+    const bool mine = rank_by_counting(key_of, n, S, slice_len, reinterpret_cast<uint64_t*>(smem_raw), s_cnt, &cnt);
+    if (mine) rank[(int64_t)b * n + blockIdx.x * kRankThreads + threadIdx.x] = cnt;
+    // every key is looked at by the CTAs of slice 0 as "their own" key: one report is enough
+    if (nonfinite && blockIdx.y == 0 && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
 }
 
 // One CTA per sequence: the kept tokens in ascending order (prefix sum of rank < k over the index) and
@@ -133,36 +90,15 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
     if (score_stride == 0) score_stride = n;
     if (score_stride < n) return LVLM_ERR_INVALID_ARG;
     if (n > kMaxSortN) return LVLM_ERR_UNSUPPORTED;
-    const int jblocks = (n + kSelThreads - 1) / kSelThreads;
-    // slices: up to eight CTAs of 256 threads per SM, at least 256 keys per slice
-    int S = 1;
-    while (S < kSelMaxCluster && (int64_t)jblocks * B * (2 * S) <= 8 * 148 && n / (2 * S) >= 256) S *= 2;
-    int slice_len = (n + S - 1) / S;
-    slice_len = (slice_len + 1) & ~1;
-    const size_t smem = (size_t)slice_len * 8;
+    int S, slice_len;
+    rank_shape(n, B, &S, &slice_len);
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_count_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    // clusters along y need a launch of their own shape: grid (jblocks, S, B), cluster (1, S, 1)
     {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(jblocks, S, B);
-        cfg.blockDim = dim3(kSelThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[2];
-        int na = 0;
-        attr[na].id = cudaLaunchAttributeClusterDimension;
-        attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = (unsigned)S; attr[na].val.clusterDim.z = 1;
-        ++na;
-        if (pdl_enabled()) {
-            attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[na].val.programmaticStreamSerializationAllowed = 1;
-            ++na;
-        }
-        cfg.attrs = attr;
-        cfg.numAttrs = na;
-        LVLM_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, select_count_kernel, score, score_stride, n, S, slice_len,
-                                               rank, dev_status));
+        const lvlm_status st = launch_kernel_cluster(select_count_kernel, dim3((n + kRankThreads - 1) / kRankThreads, S, B),
+                                                     dim3(kRankThreads), (size_t)slice_len * 8, stream, dim3(1, S, 1),
+                                                     score, score_stride, n, S, slice_len, rank, dev_status);
+        if (st != LVLM_OK) return st;
     }
     if (!kept_idx && !near_tie) return LVLM_OK;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_aux_kernel,
