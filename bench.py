@@ -125,15 +125,18 @@ def bench_prefill(w, device, steps, warmup, flush, peaks, breakdown=True):
     if breakdown:
         for s, st in enumerate(run.stages):
             hidden_in = run.hidden0 if s == 0 else run.stages[s - 1].hidden_out
-            t_sc, _ = timed(lambda: st.run_score(run.Q[s], run.K[s]), steps, warmup, flush,
-                            between=run.restore)
-            t_se, _ = timed(st.run_select, steps, warmup, flush)
-            t_me, _ = timed(lambda: st.run_merge(hidden_in, run.K[s], run.V[s], run.pos[s]),
-                            steps, warmup, flush, between=run.restore)
+            # every call captured in a graph of its own, so that no host time is measured
+            g_sc = P.capture(lambda: st.run_score(run.Q[s], run.K[s]))
+            g_se = P.capture(st.run_select)
+            g_me = P.capture(lambda: st.run_merge(hidden_in, run.K[s], run.V[s], run.pos[s]))
+            run.restore()
+            t_sc, _ = timed(g_sc.replay, steps, warmup, flush, between=run.restore)
+            t_se, _ = timed(g_se.replay, steps, warmup, flush)
+            t_me, _ = timed(g_me.replay, steps, warmup, flush, between=run.restore)
             by = st.bytes_merge_hidden() + st.bytes_merge_kv()
             res["stages"].append({
                 "n_in": st.n, "n_out": st.M, "score_ms": t_sc, "select_ms": t_se,
-                "merge_compact_ms": t_me, "merge_compact_bytes": by,
+                "merge_compact_ms": t_me, "merge_compact_bytes": by, "score_flops": st.flops_score(),
                 "merge_compact_gbs": by / (t_me * 1e6),
                 "merge_compact_frac_hbm": by / (t_me * 1e6) / peaks["hbm_gbs"],
                 "score_tflops": st.flops_score() / (t_sc * 1e9),
@@ -144,8 +147,10 @@ def bench_prefill(w, device, steps, warmup, flush, peaks, breakdown=True):
         nk = P.ReduceStage(st0.B, st0.N, st0.C, st0.H, st0.Hkv, st0.cap, st0.i0, st0.n, st0.M, device,
                            mode=L.W_NEAREST_KEPT)
         nk.rank.copy_(st0.rank)
-        t_nk, _ = timed(lambda: nk.run_merge(run.hidden0, run.K[0], run.V[0], run.pos[0]), steps, warmup, flush,
-                        between=run.restore)
+        g_nk = P.capture(lambda: nk.run_merge(run.hidden0, run.K[0], run.V[0], run.pos[0]))
+        run.restore()
+        t_nk, _ = timed(g_nk.replay, steps, warmup, flush, between=run.restore)
+        del g_nk
         res["nearest_kept_stage1"] = {"merge_compact_ms": t_nk, "similarity_flops": nk.flops_similarity(),
                                       "tflops_over_whole_call": nk.flops_similarity() / (t_nk * 1e9),
                                       "frac_tensor_over_whole_call": nk.flops_similarity() / (t_nk * 1e9) / peaks["bf16_tflops"]}
@@ -192,13 +197,25 @@ class FullPass:
         self.e_lo = torch.full(((w.L - first) * w.B,), w.i0, dtype=torch.int32, device=device)
         self.e_hi = torch.tensor([self.lens[l] - w.T for l in range(first, w.L) for _ in range(w.B)],
                                  dtype=torch.int32, device=device)
-        self.ws_sc, self.sc = [], []
-        for l in range(w.L):
-            Nl = self.lens[l]
-            d = L.Dims(B=w.B, H=w.H, Hkv=w.Hkv, D=128, N=Nl, cap=cap, i0=0, n=Nl, q_lo=Nl - w.T,
+        # after prefill every layer's text-window queries and keys exist, so the layers whose caches
+        # have the same length are scored in one call (the layer index folds into the batch)
+        self.groups = []
+        l = first
+        while l < w.L:
+            l1 = l
+            while l1 < w.L and self.lens[l1] == self.lens[l]:
+                l1 += 1
+            Nl, nb = self.lens[l], (l1 - l) * w.B
+            d = L.Dims(B=nb, H=w.H, Hkv=w.Hkv, D=128, N=Nl, cap=cap, i0=0, n=Nl, q_lo=Nl - w.T,
                        q_hi=Nl, causal=1)
-            self.ws_sc.append(L.alloc_workspace(L.OP_SCORE_TOKENS, d, device))
-            self.sc.append(torch.empty(w.B, Nl, dtype=torch.float32, device=device))
+            self.groups.append({
+                "l0": l, "l1": l1, "N": Nl,
+                "Q": torch.cat(self.Qwin[l:l1], 0).contiguous(),
+                "K": self.dec.K[l:l1].view(nb, w.Hkv, cap, 128),
+                "head": self.dec.acc[l:l1].view(nb, w.Hkv, cap)[:, :, :Nl],
+                "score": torch.empty(nb, Nl, dtype=torch.float32, device=device),
+                "ws": L.alloc_workspace(L.OP_SCORE_TOKENS, d, device)})
+            l = l1
         self.q_dec, self.k_new, self.v_new = [
             torch.stack(t) for t in zip(*[tuple(x[0] for x in I.decode_inputs(w, l, 0, 1, device))
                                           for l in range(w.L)])]
@@ -211,13 +228,16 @@ class FullPass:
     def phase_reduce(self):
         self.pre.step()
 
-    def phase_compress(self):
+    def phase_score_caches(self):
         w, L = self.w, self.L
-        for l in range(self.first, w.L):
-            Nl = self.lens[l]
-            L.score_tokens(self.Qwin[l], self.dec.K[l], N=Nl, i0=0, n=Nl, q_lo=Nl - w.T, q_hi=Nl,
-                           causal=True, score_out=self.sc[l], head_out=self.dec.acc[l][:, :, :Nl],
-                           ws=self.ws_sc[l])
+        for g in self.groups:
+            Nl = g["N"]
+            L.score_tokens(g["Q"], g["K"], N=Nl, i0=0, n=Nl, q_lo=Nl - w.T, q_hi=Nl, causal=True,
+                           score_out=g["score"], head_out=g["head"], ws=g["ws"])
+
+    def phase_compress(self):
+        w = self.w
+        self.phase_score_caches()
         self.dec.compress(beta=w.beta, e_lo=self.e_lo, e_hi=self.e_hi, first_layer=self.first)
 
     def phase_decode(self):
@@ -233,7 +253,7 @@ class FullPass:
         w = self.w
         # reduction stages; 2 scoring kernels per compressed layer + plan and compaction; one decode
         # kernel per layer
-        return self.pre.launches + 2 * (w.L - self.first) + 2 + w.L
+        return self.pre.launches + 2 * len(self.groups) + 2 + w.L
 
 
 def bench_full(w, device, steps, warmup, flush, peaks, phases=True):
@@ -249,6 +269,8 @@ def bench_full(w, device, steps, warmup, flush, peaks, phases=True):
     t_red, _ = timed(g_red.replay, steps, warmup, flush, between=fp.restore)
     g_cmp = P.capture(fp.phase_compress); fp.restore()
     t_cmp, _ = timed(g_cmp.replay, steps, warmup, flush, between=fp.restore)
+    g_scc = P.capture(fp.phase_score_caches); fp.restore()
+    t_scc, _ = timed(g_scc.replay, steps, warmup, flush, between=fp.restore)
     fp.restore(); fp.phase_compress(); torch.cuda.synchronize()
     lens_after = fp.dec.len.clone()
     Kc, Vc = fp.dec.K.clone(), fp.dec.V.clone()
@@ -261,7 +283,13 @@ def bench_full(w, device, steps, warmup, flush, peaks, phases=True):
     t_dec, _ = timed(g_dec.replay, steps, warmup, flush, between=restore_after_compress)
     kv_bytes = (int(lens_after.sum().item()) + w.L * w.B * w.Hkv) * 128 * 2 * 2
     kept = lens_after[fp.first:].float().mean().item()
+    # what the compression itself has to move: K and V rows read once and the survivors written, scores
+    lens_before = fp.len0[fp.first:].sum().item()
+    cmp_bytes = (lens_before + int(lens_after[fp.first:].sum().item())) * 128 * 2 * 2 + lens_before * 8
+    scc_flops = sum(2.0 * 2 * w.T * g["N"] * 128 * w.H * g["Q"].shape[0] for g in fp.groups)
     res = {"ms_per_step": ms, "reduce_ms": t_red, "compress_ms": t_cmp, "decode_ms": t_dec,
+           "score_caches_ms": t_scc, "score_caches_flops": scc_flops, "score_caches_calls": len(fp.groups),
+           "kv_compress_only_ms": max(t_cmp - t_scc, 0.0), "kv_compress_bytes": int(cmp_bytes),
            "tokens_in": fp.pre.tokens_in, "launches": fp.launches,
            "decode_kv_bytes": kv_bytes, "decode_gbs": kv_bytes / (t_dec * 1e6),
            "decode_frac_hbm": kv_bytes / (t_dec * 1e6) / peaks["hbm_gbs"],
@@ -510,12 +538,39 @@ def main():
     for s, st in enumerate(stage_break["stages"]):
         calls += [(f"stage{s + 1}.score", st["score_ms"]), (f"stage{s + 1}.select", st["select_ms"]),
                   (f"stage{s + 1}.merge_compact", st["merge_compact_ms"])]
-    s1 = stage_break["stages"][0]
-    roofline = {"bound": "hbm", "kernel": "lvlm_merge_compact (stage 1: hidden out of place, K and V in place)",
-                "achieved": s1["merge_compact_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": s1["merge_compact_frac_hbm"], "traffic": None,
-                "peak_source": peaks["source"], "algorithmic_bytes": s1["merge_compact_bytes"],
-                "ms": s1["merge_compact_ms"]}
+    # the step by kind of call: time per step, launches, and the roofline that bounds the kind
+    st_all = stage_break["stages"]
+    n_st = len(st_all)
+    kinds = {
+        "lvlm_score_tokens": {
+            "bound": "tensor", "unit": "TFLOP/s", "peak": peaks["bf16_tflops"],
+            "ms": sum(x["score_ms"] for x in st_all) + res["score_caches_ms"],
+            "work": sum(x["score_flops"] for x in st_all) + res["score_caches_flops"],
+            "calls": n_st + res["score_caches_calls"], "launches": 2 * (n_st + res["score_caches_calls"])},
+        "lvlm_merge_compact": {
+            "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+            "ms": sum(x["merge_compact_ms"] for x in st_all), "work": sum(x["merge_compact_bytes"] for x in st_all),
+            "calls": n_st, "launches": 3 * n_st},
+        "lvlm_kv_compress": {
+            "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"], "ms": res["kv_compress_only_ms"],
+            "work": res["kv_compress_bytes"], "calls": 1, "launches": 2},
+        "lvlm_decode_attn": {
+            "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"], "ms": res["decode_ms"],
+            "work": res["decode_kv_bytes"], "calls": w.L, "launches": w.L},
+    }
+    rooflines = {}
+    for name, kd in kinds.items():
+        ach = kd["work"] / (kd["ms"] * (1e9 if kd["bound"] == "tensor" else 1e6)) if kd["ms"] > 0 else 0.0
+        rooflines[name] = {"bound": kd["bound"], "achieved": ach, "peak": kd["peak"], "unit": kd["unit"],
+                           "frac": ach / kd["peak"], "traffic": None, "ms_per_step": kd["ms"],
+                           "ms_per_call": kd["ms"] / kd["calls"], "calls_per_step": kd["calls"],
+                           "launches_per_step": kd["launches"],
+                           "algorithmic_work_per_call": kd["work"] / kd["calls"]}
+    rooflines["lvlm_select_topk"] = {"bound": "latency", "ms_per_step": sum(x["select_ms"] for x in st_all),
+                                     "calls_per_step": n_st, "launches_per_step": n_st}
+    dominant = max(kinds, key=lambda k: kinds[k]["ms"])
+    roofline = dict(rooflines[dominant], kernel=dominant, peak_source=peaks["source"] + " (of measured)"
+                    if peaks["source"] == "measured" else peaks["source"] + " (of fallback)")
     out = {
         "metric": "reduced image tokens/s", "value": value, "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
@@ -532,7 +587,7 @@ def main():
         "decode": {"value": res["decode_gbs"], "unit": "GB/s", "frac_of_hbm_peak": res["decode_frac_hbm"],
                    "kv_bytes_per_step": res["decode_kv_bytes"],
                    "mean_len_after_compress": res["mean_len_after_compress"]},
-        "roofline": roofline, "clocks": clocks, "gpu_launches": res["launches"] * args.steps,
+        "roofline": roofline, "rooflines": rooflines, "clocks": clocks, "gpu_launches": res["launches"] * args.steps,
         "peaks": peaks,
     }
     if rank == 0 and world == 1:
