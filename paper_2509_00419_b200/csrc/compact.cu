@@ -53,6 +53,7 @@ __device__ __forceinline__ float ld_cluster_f32(const float* my_smem, uint32_t r
 }
 
 // grid.x = column groups * S (clusters of S along x), grid.y = G (* 2 with a second tensor), grid.z = B
+template <int MAXC>                                      // 16-byte column groups per thread
 __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const InplaceArgs a) {
     extern __shared__ __align__(16) uint4 tile[];
     pdl_enter();
@@ -85,9 +86,9 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
     int32_t* s_idx = reinterpret_cast<int32_t*>(tile + 2 * (size_t)a.Rmax * a.Vsub);     // [3][Rmax]
     constexpr int kIdxPerThread = 2;                     // Rmax <= 2 * blockDim.x
 
-    float acc[kCompactMaxC][8];
+    float acc[MAXC][8];
 #pragma unroll
-    for (int ci = 0; ci < kCompactMaxC; ++ci)
+    for (int ci = 0; ci < MAXC; ++ci)
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
 
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
             const int sidx = s_idx[slot * a.Rmax + rr];
             if (sidx >= 0) {
 #pragma unroll
-                for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                for (int ci = 0; ci < MAXC; ++ci) {
                     const int c = cg + ci * CG;
                     if (c < vw) cp_async16(&dst[rr * a.Vsub + c], rows + (int64_t)sidx * V + c);
                 }
@@ -142,7 +143,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
             // merged rows inside my positions: read before anyone overwrites them; four rows in flight
             for (int rb = rl; rb < R; rb += 4 * RL) {
                 float wj[4];
-                uint4 x[4][kCompactMaxC];
+                uint4 x[4][MAXC];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int rr = rb + u * RL;
@@ -153,7 +154,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
                 for (int u = 0; u < 4; ++u) {
                     const int o = t0 + rank * R + rb + u * RL;
 #pragma unroll
-                    for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                    for (int ci = 0; ci < MAXC; ++ci) {
                         const int c = cg + ci * CG;
                         x[u][ci] = (wj[u] != 0.f && c < vw) ? rows[(int64_t)o * V + c] : make_uint4(0, 0, 0, 0);
                     }
@@ -162,7 +163,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
                 for (int u = 0; u < 4; ++u) {
                     if (wj[u] != 0.f) {
 #pragma unroll
-                        for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                        for (int ci = 0; ci < MAXC; ++ci) {
                             const uint4 xv = x[u][ci];
                             acc[ci][0] = fmaf(wj[u], bf16_lo(xv.x), acc[ci][0]); acc[ci][1] = fmaf(wj[u], bf16_hi(xv.x), acc[ci][1]);
                             acc[ci][2] = fmaf(wj[u], bf16_lo(xv.y), acc[ci][2]); acc[ci][3] = fmaf(wj[u], bf16_hi(xv.y), acc[ci][3]);
@@ -181,7 +182,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
             if (cur_idx[rr] >= 0) {
                 const int o = t0 + rank * R + rr;
 #pragma unroll
-                for (int ci = 0; ci < kCompactMaxC; ++ci) {
+                for (int ci = 0; ci < MAXC; ++ci) {
                     const int c = cg + ci * CG;
                     if (c < vw) rows[(int64_t)o * V + c] = cur[rr * a.Vsub + c];
                 }
@@ -195,7 +196,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
     // merged row: row lanes added in lane order, CTAs in rank order, rounded once, stored by rank 0
     float* red = reinterpret_cast<float*>(tile);          // [RL][vw][8]
 #pragma unroll
-    for (int ci = 0; ci < kCompactMaxC; ++ci) {
+    for (int ci = 0; ci < MAXC; ++ci) {
         const int c = cg + ci * CG;
         if (c < vw) {
 #pragma unroll
@@ -262,10 +263,18 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
     const size_t red = ((size_t)a.RL + 1) * Vsub * 32;
     if (red > smem) smem = red;
     if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
-    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(inplace_compact_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    return launch_kernel(inplace_compact_kernel, dim3((unsigned)(ncol * S), (unsigned)(G * (base1 ? 2 : 1)), (unsigned)B),
-                         dim3(kCompactThreads), smem, stream, S, a);
+    const dim3 grid((unsigned)(ncol * S), (unsigned)(G * (base1 ? 2 : 1)), (unsigned)B);
+    const int chunks = (Vsub + CG - 1) / CG;
+#define LVLM_COMPACT_CASE(MC)                                                                              \
+    do {                                                                                                   \
+        LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(inplace_compact_kernel<MC>,                               \
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem)); \
+        return launch_kernel(inplace_compact_kernel<MC>, grid, dim3(kCompactThreads), smem, stream, S, a); \
+    } while (0)
+    if (chunks <= 1) LVLM_COMPACT_CASE(1);
+    if (chunks <= 2) LVLM_COMPACT_CASE(2);
+    LVLM_COMPACT_CASE(4);
+#undef LVLM_COMPACT_CASE
 }
 
 }  // namespace lvlm
