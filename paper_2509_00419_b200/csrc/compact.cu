@@ -140,18 +140,19 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
         int reg[kIdxPerThread];
         fetch_idx(t0 + 2 * Rc, reg);                  // in flight while this round runs
         if (w) {
-            // merged rows inside my positions: read before anyone overwrites them; four rows in flight
-            for (int rb = rl; rb < R; rb += 4 * RL) {
-                float wj[4];
-                uint4 x[4][MAXC];
+            // merged rows inside my positions: read before anyone overwrites them; kWB rows in flight
+            constexpr int kWB = 16 / MAXC;
+            for (int rb = rl; rb < R; rb += kWB * RL) {
+                float wj[kWB];
+                uint4 x[kWB][MAXC];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kWB; ++u) {
                     const int rr = rb + u * RL;
                     const int o = t0 + rank * R + rr;
                     wj[u] = (rr < R && o < Nscan && o >= a.i0 && o < a.i0 + a.n) ? w[o - a.i0] : 0.f;
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kWB; ++u) {
                     const int o = t0 + rank * R + rb + u * RL;
 #pragma unroll
                     for (int ci = 0; ci < MAXC; ++ci) {
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kWB; ++u) {
                     if (wj[u] != 0.f) {
 #pragma unroll
                         for (int ci = 0; ci < MAXC; ++ci) {
