@@ -34,6 +34,7 @@ struct ScoreTcArgs {
     const float* lse_user;     // natural-log row normalisers from the caller, or NULL
     float* lse_ws;             // [B][H][Nq] log2-domain normalisers (pass 1 writes, pass 2 reads)
     float* partial;            // [B][Hkv * hsplit][n] column sums of each CTA row (pass 2 writes)
+    int ksplit;                // pass 1: CTAs (one cluster) that share the key tiles of a query tile
     int nkt;                   // key tiles of pass 2 (its grid.x)
     int hsplit;                // CTAs that share the query heads of one KV group in pass 2
     int32_t* cnt;              // [B][key tiles] CTAs of pass 2 that have parked their sums (zero at its start)
@@ -51,6 +52,18 @@ struct TcSmem {
     float lse_s[8][2][kTile / 2];  // per epilogue warp, per accumulator buffer: normalisers of its 64 columns
     float xm[kTile], xl[kTile];    // what the warps of the upper column half hand to the lower half
 };
+
+__device__ __forceinline__ void cluster_barrier_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(const float* my_smem, uint32_t rank) {
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, TcSmem* sm, int32_t* dev_status) {
     if (sm->abort) return false;
@@ -78,11 +91,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     // ---- which tiles this CTA multiplies ---------------------------------------------------------
     int nt, h = 0, g = 0, qt = 0, kt = 0, qt_min = 0, nqt_vis = 0;
     const int h_first = MODE == 1 ? (blockIdx.y / a.hsplit) * a.G + (blockIdx.y % a.hsplit) * (a.G / a.hsplit) : 0;
+    int t_off = 0;                                        // pass 1: first key tile of this CTA
     if (MODE == 0) {
-        qt = blockIdx.x; h = blockIdx.y; g = h / a.G;
+        qt = blockIdx.x / a.ksplit; h = blockIdx.y; g = h / a.G;
         const int last_pos = a.q_lo + min(a.Nq, (qt + 1) * kTile) - 1;
         const int key_end = a.causal ? min(a.N, last_pos + 1) : a.N;
-        nt = (key_end + kTile - 1) / kTile;
+        const int nt_all = (key_end + kTile - 1) / kTile;
+        const int per = (nt_all + a.ksplit - 1) / a.ksplit;
+        t_off = min(nt_all, (int)(blockIdx.x % a.ksplit) * per);
+        nt = min(nt_all, t_off + per) - t_off;
     } else {
         kt = blockIdx.x; g = blockIdx.y / a.hsplit;
         const int j0 = a.i0 + kt * kTile;
@@ -127,8 +144,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
                 unsigned char* dst = sB + st * kTileBytes;
                 mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
                 if (MODE == 0) {
-                    tma_load_4d(dst, &kmap, &sm->full[st], 0, t * kTile, g, b);
-                    tma_load_4d(dst + kHalfBytes, &kmap, &sm->full[st], 64, t * kTile, g, b);
+                    tma_load_4d(dst, &kmap, &sm->full[st], 0, (t_off + t) * kTile, g, b);
+                    tma_load_4d(dst + kHalfBytes, &kmap, &sm->full[st], 64, (t_off + t) * kTile, g, b);
                 } else {
                     const int hh = h_first + t / nqt_vis, q2 = qt_min + t % nqt_vis;
                     tma_load_4d(dst, &qmap, &sm->full[st], 0, hh, q2 * kTile, b);
@@ -204,7 +221,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
                 tmem_ld32(lane_addr + buf * kTile + c4 * 32, v);
                 tmem_ld_wait();
                 if (MODE == 0) {
-                    const int jb = t * kTile + c4 * 32;
+                    const int jb = (t_off + t) * kTile + c4 * 32;
                     const int lim = min(a.N, a.causal ? my_pos + 1 : a.N) - jb;    // columns < lim are visible
                     float cmax = -INFINITY;
 #pragma unroll
@@ -247,7 +264,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
                 if (m_run > -INFINITY) L += l_run * exp2f(m_run - M);
                 if (m1 > -INFINITY) L += l1 * exp2f(m1 - M);
                 const int i = qt * kTile + row;
-                if (!sm->abort && i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = M + log2f(L);
+                if (a.ksplit == 1) {
+                    if (!sm->abort && i < a.Nq) a.lse_ws[((int64_t)b * a.H + h) * a.Nq + i] = M + log2f(L);
+                } else {                                   // the cluster combines below
+                    sm->xm[row] = M; sm->xl[row] = L;
+                }
             }
         } else {
             if (half == 0) colsum += sm->xm[row];
@@ -282,6 +303,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     // ---- common exit: everyone meets, then the allocating warp frees the tensor memory ----------
     tc_fence_before();
     __syncthreads();
+    if (MODE == 0 && a.ksplit > 1) {
+        // the CTAs of the cluster hold (max, sum) of their share of the keys for the same 128 rows:
+        // rank 0 adds them in rank order and writes the normalisers
+        cluster_barrier_all();
+        if (blockIdx.x % a.ksplit == 0 && threadIdx.x >= 64 && threadIdx.x < 64 + kTile) {
+            const int row = threadIdx.x - 64;
+            float M = -INFINITY;
+            for (int r = 0; r < a.ksplit; ++r) M = fmaxf(M, ld_cluster_f32(&sm->xm[row], r));
+            float L = 0.f;
+            for (int r = 0; r < a.ksplit; ++r) {
+                const float m = ld_cluster_f32(&sm->xm[row], r);
+                if (m > -INFINITY) L += ld_cluster_f32(&sm->xl[row], r) * exp2f(m - M);
+            }
+            const int i = (blockIdx.x / a.ksplit) * kTile + row;
+            if (!sm->abort && i < a.Nq) a.lse_ws[((int64_t)b * a.H + blockIdx.y) * a.Nq + i] = M + log2f(L);
+        }
+        cluster_barrier_all();
+    }
     if (sm->abort) {                              // let copies still in flight land before leaving
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
@@ -325,13 +364,18 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
         hsplit = hs;
         if ((int64_t)nkt * d->Hkv * d->B * hs >= 148) break;
     }
-    a.hsplit = hsplit; a.nkt = nkt;
+    a.hsplit = hsplit; a.nkt = nkt; a.ksplit = 1;
     if (lse) LVLM_RETURN_IF_CUDA(cudaMemsetAsync(cnt, 0, (size_t)d->B * nkt * 4, stream));
     if (!lse) {
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<0>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        const lvlm_status s0 = launch_kernel(score_tc_kernel<0>, dim3(nqt, d->H, d->B), dim3(kTcThreads), smem,
-                                             stream, 1, qmap, kmap, a);
+        // pass 1: when query tiles x heads do not fill the GPU, a cluster of CTAs shares the key tiles
+        int ksplit = 1;
+        const int max_kt = (d->N + kTile - 1) / kTile;
+        while (ksplit < 8 && (int64_t)nqt * d->H * d->B * ksplit < 148 && 2 * ksplit <= max_kt) ksplit *= 2;
+        a.ksplit = ksplit;
+        const lvlm_status s0 = launch_kernel(score_tc_kernel<0>, dim3(nqt * ksplit, d->H, d->B), dim3(kTcThreads),
+                                             smem, stream, ksplit, qmap, kmap, a);
         if (s0 != LVLM_OK) return s0;
     }
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<1>,
