@@ -65,6 +65,57 @@ __device__ __forceinline__ float ld_cluster_f32(const float* my_smem, uint32_t r
     return v;
 }
 
+// 2^x on the special-function unit, one instruction (2 ulp, flush to zero: the scores tolerate 1e-3).
+__device__ __forceinline__ float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Pass 1, one chunk of 32 raw logits of a query row: columns [0, lim) are visible.  Updates the running
+// (max, sum of 2^(logit*scale - max)).  Four partial sums keep the adds off one dependency chain.
+__device__ __forceinline__ void rowstat_chunk(float* v, int lim, float scale_log2, float& m_run, float& l_run) {
+    float cmax = -INFINITY;
+    if (lim >= 32) {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) { v[c] *= scale_log2; cmax = fmaxf(cmax, v[c]); }
+    } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) { v[c] = c < lim ? v[c] * scale_log2 : -INFINITY; cmax = fmaxf(cmax, v[c]); }
+    }
+    const float m_new = fmaxf(m_run, cmax);
+    if (m_new > -INFINITY) {
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+            s0 += ex2_fast(v[c] - m_new); s1 += ex2_fast(v[c + 1] - m_new);
+            s2 += ex2_fast(v[c + 2] - m_new); s3 += ex2_fast(v[c + 3] - m_new);
+        }
+        l_run = l_run * ex2_fast(m_run - m_new) + ((s0 + s1) + (s2 + s3));
+        m_run = m_new;
+    }
+}
+
+// Pass 2, one chunk of 32 raw logits of a key against 32 query rows with normalisers ls (log2 domain):
+// sum of the probabilities of the rows c >= first.
+__device__ __forceinline__ float colsum_chunk(const float* v, const float* ls, int first, float scale_log2) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    if (first <= 0) {
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+            s0 += ex2_fast(fmaf(v[c], scale_log2, -ls[c])); s1 += ex2_fast(fmaf(v[c + 1], scale_log2, -ls[c + 1]));
+            s2 += ex2_fast(fmaf(v[c + 2], scale_log2, -ls[c + 2])); s3 += ex2_fast(fmaf(v[c + 3], scale_log2, -ls[c + 3]));
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const float p = ex2_fast(fmaf(v[c], scale_log2, -ls[c]));
+            s0 += c >= first ? p : 0.f;
+        }
+    }
+    return (s0 + s1) + (s2 + s3);
+}
+
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, TcSmem* sm, int32_t* dev_status) {
     if (sm->abort) return false;
     if (mbar_wait(bar, parity)) return true;
@@ -223,30 +274,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
                 if (MODE == 0) {
                     const int jb = (t_off + t) * kTile + c4 * 32;
                     const int lim = min(a.N, a.causal ? my_pos + 1 : a.N) - jb;    // columns < lim are visible
-                    float cmax = -INFINITY;
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        v[c] = c < lim ? v[c] * a.scale_log2 : -INFINITY;
-                        cmax = fmaxf(cmax, v[c]);
-                    }
-                    const float m_new = fmaxf(m_run, cmax);
-                    if (m_new > -INFINITY) {
-                        float add = 0.f;
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) add += exp2f(v[c] - m_new);
-                        l_run = l_run * exp2f(m_run - m_new) + add;
-                        m_run = m_new;
-                    }
+                    rowstat_chunk(v, lim, a.scale_log2, m_run, l_run);
                 } else {
                     const int ib = q2 * kTile + c4 * 32;                           // first query row of the chunk
                     // query i sees my key iff my_key <= q_lo + i  <=>  c >= my_key - q_lo - ib
                     const int first = a.causal ? my_key - a.q_lo - ib : 0;
-                    const float* ls = &sm->lse_s[warp - 2][buf][c2 * 32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float p = exp2f(v[c] * a.scale_log2 - ls[c]);
-                        colsum += c >= first ? p : 0.f;
-                    }
+                    colsum += colsum_chunk(v, &sm->lse_s[warp - 2][buf][c2 * 32], first, a.scale_log2);
                 }
             }
             tc_fence_before();
