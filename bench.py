@@ -430,35 +430,35 @@ def cpu_baseline(w):
 
 # ------------------------------------------------------------------------------------------
 def e2e_pass(w, device, steps, warmup):
-    """The reduction stages through the public API with HOST buffers: every step copies the
-    stage inputs from pinned host memory, runs the calls, and reads the result back."""
-    from paper_2509_00419_b200 import pipeline as P
-    run = P.PyramidPrefill(w, device)
-    host = {"hidden": run.hidden0.cpu().pin_memory(),
-            "Q": [t.cpu().pin_memory() for t in run.Q], "K": [t.cpu().pin_memory() for t in run.K0],
-            "V": [t.cpu().pin_memory() for t in run.V0], "pos": [t.cpu().pin_memory() for t in run.pos0]}
-    last = run.stages[-1]
-    out_host = torch.empty(last.hidden_out.shape, dtype=torch.bfloat16).pin_memory()
-    len_host = torch.empty(w.B, dtype=torch.int32).pin_memory()
-    h2d = host["hidden"].numel() * 2 + sum(t.numel() * t.element_size() for k in ("Q", "K", "V", "pos")
-                                            for t in host[k])
-    d2h = out_host.numel() * 2 + len_host.numel() * 4
+    """The whole step through the public API with HOST buffers: every step copies all inputs of
+    the step from pinned host memory (hidden states, the stages' Q windows, K, V and position ids, the
+    caches and lengths of all layers, their text-window queries, the decode queries and new rows), runs
+    the calls, and reads the results back (reduced hidden states, decode outputs, cache lengths)."""
+    fp = FullPass(w, device)
+    pre = fp.pre
+    dev_in = [pre.hidden0] + pre.Q + pre.K + pre.V + pre.pos + [fp.dec.K, fp.dec.V, fp.dec.len] + \
+             [g["Q"] for g in fp.groups] + [fp.q_dec, fp.k_new, fp.v_new]
+    fp.restore()
+    torch.cuda.synchronize()
+    host_in = [t.cpu().pin_memory() for t in dev_in]
+    last = pre.stages[-1]
+    dev_out = [last.hidden_out, last.new_len, fp.dec.out, fp.dec.len]
+    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in dev_out]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
 
     def step():
-        run.hidden0.copy_(host["hidden"], non_blocking=True)
-        for s in range(len(run.stages)):
-            run.Q[s].copy_(host["Q"][s], non_blocking=True)
-            run.K[s].copy_(host["K"][s], non_blocking=True)
-            run.V[s].copy_(host["V"][s], non_blocking=True)
-            run.pos[s].copy_(host["pos"][s], non_blocking=True)
-        run.step()
-        out_host.copy_(last.hidden_out, non_blocking=True)
-        len_host.copy_(last.new_len, non_blocking=True)
+        for dt, ht in zip(dev_in, host_in):
+            dt.copy_(ht, non_blocking=True)
+        fp.dec.acc.zero_()
+        fp.step()
+        for ht, dt in zip(host_out, dev_out):
+            ht.copy_(dt, non_blocking=True)
 
     ms, _ = timed(step, steps, warmup, None)
-    return {"value": run.tokens_in / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
+    return {"value": pre.tokens_in / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-            "what": "reduction stages of the headline workload, inputs from pinned host memory"}
+            "what": "the whole step through the Python binding of the C ABI, inputs from pinned host memory, results read back"}
 
 
 # ------------------------------------------------------------------------------------------
