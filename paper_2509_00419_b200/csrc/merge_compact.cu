@@ -193,6 +193,13 @@ __device__ __forceinline__ void hid_cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n"
                  "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
+__device__ __forceinline__ int hid_ld_cluster_i32(const int* my_smem, uint32_t rank) {
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    int v;
+    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+    return v;
+}
 __device__ __forceinline__ float4 hid_ld_cluster_f4(const float* my_smem, uint32_t rank) {
     uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
@@ -309,49 +316,65 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
             }
         }
     }
-    hid_cluster_barrier();                                    // rank 0 has read every CTA's sums
-    if (rank != 0) return;
-    // ---- the last cluster of this sequence finalises P_new ------------------------------------------------
+    // ---- the last cluster of this sequence finalises P_new, all of its CTAs sharing the columns -----------
+    if (rank == 0) {
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const int ticket = atomicAdd(&meta[b * kMetaInts + 1], 1);
+            s_last = ticket == q_last - q_first;
+        }
+    }
+    hid_cluster_barrier();                 // rank 0 has read every CTA's sums and knows whether we are last
+    const int last = cl > 1 ? hid_ld_cluster_i32(&s_last, 0) : s_last;
+    hid_cluster_barrier();                 // ... and everybody has asked it
+    if (!last) return;
     __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int ticket = atomicAdd(&meta[b * kMetaInts + 1], 1);
-        s_last = ticket == q_last - q_first;
+    const int nq = q_last - q_first + 1;                      // partials to add, in cluster order
+    const int Vs = (V + cl - 1) / cl;                         // my slice of the column groups
+    const int c_lo = min(V, rank * Vs), c_hi = min(V, c_lo + Vs);
+    // two threads per column group, each adding half of the partials (four in flight); the halves are
+    // added in order through shared memory
+    const int hsel = tid >> 7, lane_c = tid & 127;
+    const int q_mid = q_first + (nq + 1) / 2;
+    const int qa = hsel ? q_mid : q_first, qb = hsel ? q_last + 1 : q_mid;
+    float* s_fin = s_sum;                                     // [2][c_hi - c_lo][8], free after the barriers
+    for (int cb = c_lo; cb < c_hi; cb += 128) {
+        const int c = cb + lane_c;
+        float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (c < c_hi) {
+            for (int q = qa; q < qb; q += 4) {
+                float4 lo[4], hi[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    lo[u] = hi[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q + u < qb) {
+                        const float4* pp = reinterpret_cast<const float4*>(
+                            partial + ((int64_t)b * gridDim.x / cl + q + u) * V * 8 + c * 8);
+                        lo[u] = __ldcg(pp); hi[u] = __ldcg(pp + 1);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    t[0] += lo[u].x; t[1] += lo[u].y; t[2] += lo[u].z; t[3] += lo[u].w;
+                    t[4] += hi[u].x; t[5] += hi[u].y; t[6] += hi[u].z; t[7] += hi[u].w;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s_fin[(hsel * Vs + (c - c_lo)) * 8 + e] = t[e];
+        }
     }
     __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-#pragma unroll 1
-    for (int ci = 0; ci < CH; ++ci) {
-        const int c = tid + ci * kHidThreads;
-        if (c >= V) break;
-        float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        int q = q_first;
-        for (; q + 3 <= q_last; q += 4) {                     // four partials in flight
-            float4 lo[4], hi[4];
+    for (int c = c_lo + tid; c < c_hi; c += kHidThreads) {
+        float t[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)b * gridDim.x / cl + q + u) * V * 8 + c * 8);
-                lo[u] = __ldcg(p); hi[u] = __ldcg(p + 1);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                t[0] += lo[u].x; t[1] += lo[u].y; t[2] += lo[u].z; t[3] += lo[u].w;
-                t[4] += hi[u].x; t[5] += hi[u].y; t[6] += hi[u].z; t[7] += hi[u].w;
-            }
-        }
-        for (; q <= q_last; ++q) {
-            const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)b * gridDim.x / cl + q) * V * 8 + c * 8);
-            const float4 lo = __ldcg(p), hi = __ldcg(p + 1);
-            t[0] += lo.x; t[1] += lo.y; t[2] += lo.z; t[3] += lo.w;
-            t[4] += hi.x; t[5] += hi.y; t[6] += hi.z; t[7] += hi.w;
-        }
+        for (int e = 0; e < 8; ++e) t[e] = s_fin[(c - c_lo) * 8 + e] + s_fin[(Vs + (c - c_lo)) * 8 + e];
         uint4 o;
         o.x = pack_bf16(t[0], t[1]); o.y = pack_bf16(t[2], t[3]);
         o.z = pack_bf16(t[4], t[5]); o.w = pack_bf16(t[6], t[7]);
         hout[(int64_t)(i0 + k) * V + c] = o;
     }
-    if (tid == 0) meta[b * kMetaInts + 1] = 0;
+    if (rank == 0 && tid == 0) meta[b * kMetaInts + 1] = 0;
 }
 
 template <int CH>
@@ -359,7 +382,7 @@ static lvlm_status launch_hidden_stream(const void* hidden, void* hidden_out, in
                                         const lvlm_dims* d, const HiddenGrid& L, const int32_t* dst_map,
                                         const float* wgt, int32_t* meta, float* partial, void* scratch,
                                         int64_t scr_sb, cudaStream_t stream) {
-    const size_t smem = (size_t)L.V * 32;
+    const size_t smem = (size_t)L.V * 32 * (L.cl > 1 ? 1 : 2);      // the final sum needs two rows without a cluster
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(hidden_stream_kernel<CH>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     return launch_kernel(hidden_stream_kernel<CH>, dim3((unsigned)L.cps, (unsigned)d->B), dim3(kHidThreads), smem,
