@@ -121,35 +121,37 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
     }
     __syncthreads();
 
-    const int per = (n + blockDim.x - 1) / blockDim.x;
-    const int j0 = min(n, (int)threadIdx.x * per), j1 = min(n, j0 + per);
-    int cnt = 0, first_drop = n;
+    // tile by tile, thread = token of the tile (coalesced), running count of the kept tokens so far
     bool bad = false;
-    for (int j = j0; j < j1; ++j) {
-        const int rj = rk[j];
-        if (rj < 0 || rj >= n) bad = true;
-        if (rj < k) ++cnt; else if (first_drop == n) first_drop = j;
-        if (rj == k) s_merged_tok = j;
-    }
-    int total;
-    int off = block_exclusive_scan(cnt, scan_scratch, &total);
-    if (total != k) bad = true;
-    if (first_drop < n) atomicMin(&s_first_drop, first_drop);
-    for (int j = j0; j < j1; ++j) {
-        const int rj = rk[j];
-        float wj = 0.f;
-        if (rj < k) {
-            if (off < k) src[i0 + off] = i0 + j;
-            dst[i0 + j] = off < k ? i0 + off : -1;
-            ++off;
-        } else {
-            dst[i0 + j] = -1;
-            int p = rj - k;
-            p = p < 0 ? 0 : (p >= r1 ? r1 - 1 : p);
-            wj = merge_weight(mode, p, r1, inv_sum, w_custom);
+    int kept_before = 0;
+    for (int t0 = 0; t0 < n; t0 += blockDim.x) {
+        const int j = t0 + threadIdx.x;
+        const int rj = j < n ? rk[j] : n;                 // past the end: counts as dropped, writes nothing
+        if (j < n && (rj < 0 || rj >= n)) bad = true;
+        const int is_kept = j < n && rj < k;
+        int total;
+        const int off = kept_before + block_exclusive_scan(is_kept, scan_scratch, &total);
+        if (j < n) {
+            float wj = 0.f;
+            if (is_kept) {
+                if (off < k) src[i0 + off] = i0 + j;
+                dst[i0 + j] = off < k ? i0 + off : -1;
+            } else {
+                dst[i0 + j] = -1;
+                if (rj == k) s_merged_tok = j;
+                int p = rj - k;
+                p = p < 0 ? 0 : (p >= r1 ? r1 - 1 : p);
+                wj = merge_weight(mode, p, r1, inv_sum, w_custom);
+            }
+            w[j] = wj;
         }
-        w[j] = wj;
+        int fd = (j < n && !is_kept) ? j : n;              // first dropped token: one atomic per warp
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) fd = min(fd, __shfl_xor_sync(0xFFFFFFFFu, fd, o));
+        if ((threadIdx.x & 31) == 0 && fd < n) atomicMin(&s_first_drop, fd);
+        kept_before += total;
     }
+    if (kept_before != k) bad = true;
     for (int o = threadIdx.x; o < Nout; o += blockDim.x) {
         if (o < i0) { src[o] = o; dst[o] = o; }
         else if (o == i0 + k) src[o] = -1;
