@@ -330,7 +330,7 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
     dec.K.copy_(snap[0]); dec.V.copy_(snap[1]); dec.acc.copy_(snap[2]); dec.len.fill_(prompt_len)
     dec.status.zero_()
     del snap
-    t_dec, t_cmp, bytes_read, n_cmp = 0.0, 0.0, 0, 0
+    t_dec, t_cmp, bytes_read, n_cmp, moved_rows_first = 0.0, 0.0, 0, 0, 0
     cur_len = prompt_len
     for c0 in range(0, steps_total, chunk):
         ns = min(chunk, steps_total - c0)
@@ -338,6 +338,17 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
         qs, ks, vs = torch.stack(qs, 1), torch.stack(ks, 1), torch.stack(vs, 1)   # [ns, L, ...]
         evs = []
         if cur_len > w.budget:
+            if n_cmp == 0:
+                # accounting only (not on the timed path): rows a compaction really has to move are the
+                # survivors behind the first evicted entry of their head
+                ev = cur_len - w.recent
+                keep_ev = w.budget - w.recent
+                kept = torch.zeros(w.L, w.B, w.Hkv, cur_len, dtype=torch.bool, device=device)
+                kept[..., ev:] = True
+                top = dec.acc[..., :ev].topk(keep_ev, dim=-1).indices
+                kept.scatter_(-1, top, True)
+                first_drop = (~kept).float().argmax(dim=-1)
+                moved_rows_first = int((w.budget - first_drop).clamp(min=0).sum().item())
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(); g_cmp.replay(); e1.record()
             evs.append(("c", e0, e1))
@@ -364,9 +375,11 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
            "compress_us_per_layer": (t_cmp * 1e3 / (n_cmp * w.L)) if n_cmp else None,
            "final_len": cur_len, "launches": steps_total * w.L + n_cmp * 2}
     if n_cmp:
-        # bytes a compression must move per layer: read cap rows of K,V, write budget rows
-        by = w.B * w.Hkv * ((w.budget + w.trigger) + w.budget) * 128 * 2 * 2
-        res["compress_gbs"] = by * w.L * n_cmp / (t_cmp * 1e6)
+        # bytes a compression has to move: every moved row of K and V read and written once, all scores
+        # read (counted on the first compression; the later ones evict the same number of entries)
+        by = moved_rows_first * 128 * 2 * 2 * 2 + w.L * w.B * w.Hkv * (w.budget + w.trigger) * 8
+        res["compress_bytes_per_call"] = by
+        res["compress_gbs"] = by * n_cmp / (t_cmp * 1e6)
         res["compress_frac_hbm"] = res["compress_gbs"] / peaks["hbm_gbs"]
     return res
 

@@ -16,7 +16,7 @@ namespace lvlm {
 
 constexpr int kCompactThreads = 256;
 constexpr int kCompactMaxC = 4;              // 16-byte column groups per thread
-constexpr int kCompactBufBytes = 48 * 1024;  // one of the two staging buffers
+constexpr int kCompactBufBytes = 24 * 1024;  // one of the two staging buffers
 constexpr int kCompactMaxCluster = 8;
 constexpr int kCompactTargetCtas = 2 * 148;
 
@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
         fetch_idx(t0 + 2 * Rc, reg);                  // in flight while this round runs
         if (w) {
             // merged rows inside my positions: read before anyone overwrites them; kWB rows in flight
-            constexpr int kWB = 16 / MAXC;
+            constexpr int kWB = 4;
             for (int rb = rl; rb < R; rb += kWB * RL) {
                 float wj[kWB];
                 uint4 x[kWB][MAXC];
@@ -246,7 +246,7 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
     int S = 1;
     while (S < kCompactMaxCluster && nseq * (2 * S) <= kCompactTargetCtas && N / (2 * S) >= 32) S *= 2;
     int Vsub = V;
-    while (Vsub > 8 && nseq * S * ((V + Vsub - 1) / Vsub) < kCompactTargetCtas / 2) Vsub = ((Vsub + 1) / 2 + 7) / 8 * 8;
+    while (Vsub > 8 && nseq * S * ((V + Vsub - 1) / Vsub) < 2 * kCompactTargetCtas) Vsub = ((Vsub + 1) / 2 + 7) / 8 * 8;
     // rows wider than the per-thread budget are always split
     while (Vsub > kCompactMaxC * kCompactThreads) Vsub = ((Vsub + 1) / 2 + 7) / 8 * 8;
     const int ncol = (V + Vsub - 1) / Vsub;
