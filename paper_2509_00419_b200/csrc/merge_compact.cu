@@ -218,7 +218,7 @@ __device__ __forceinline__ float4 hid_ld_cluster_f4(const float* my_smem, uint32
 // order through distributed shared memory and park one partial per cluster; the last cluster of
 // the sequence to finish adds the partials in cluster order, rounds once to bf16 and writes P_new.
 template <int CH>
-__global__ void __launch_bounds__(kHidThreads)
+__global__ void __launch_bounds__(kHidThreads, CH <= 2 ? 4 : 2)     // the occupancy hidden_grid() counts on
 hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
                      int64_t hid_stride_b, int64_t out_stride_b,   // in uint4
                      int V, int N, int i0, int n, int k, int rpc, int cl,
