@@ -175,6 +175,16 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
                 }
             }
         }
+        if (w && t0 + Rc < Nscan) {
+            // the merged rows of the next round's positions start their way from DRAM now (L2 prefetch,
+            // one request per 128 bytes); nothing overwrites them before that round
+            const int lines = (vw * 16 + 127) / 128;
+            for (int e = threadIdx.x; e < R * lines; e += kCompactThreads) {
+                const int o = t0 + Rc + rank * R + e / lines;
+                if (o < Nscan && o >= a.i0 && o < a.i0 + a.n)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(rows + (int64_t)o * V + (e % lines) * 8));
+            }
+        }
         cp_async_wait_group<1>();                     // this super-tile's sources have landed
         cluster_barrier();                            // ... in every CTA of the cluster
         const uint4* cur = buf[k & 1];
