@@ -226,3 +226,28 @@ def test_nearest_kept_stage_full_size(wname, b):
     assert_rows_close(f64(out[b]), want["hidden"][0], what="merged hidden rows")
     assert_rows_close(f64(K[b, :, :st.Nout]), want["Kc"][0], what="merged K rows")
     assert_rows_close(f64(V[b, :, :st.Nout]), want["Vc"][0], what="merged V rows")
+
+
+ALL_ROWS = [("cfg1", {}), ("cfg2", {}), ("cfg3", {"B": 1}), ("cfg5", {"n": 3840, "T": 256})]
+
+
+@pytest.mark.parametrize("wname,cut", ALL_ROWS)
+def test_score_all_rows_window(wname, cut):
+    """The paper-literal importance: column sums of the whole causal attention matrix (every query row
+    of the sequence), at the configurations' sizes (cfg3 one sequence, cfg5 a 4096-token cut)."""
+    w = I.shrink(I.WORKLOADS[wname], **cut)
+    dev = torch.device("cuda", 0)
+    layer = w.stages[0][0]
+    pos = torch.arange(w.N, dtype=torch.int32, device=dev)[None].repeat(w.B, 1)
+    q, k, _ = I.layer_qkv(w, layer, pos, dev)
+    flag = torch.zeros(1, dtype=torch.int32, device=dev)
+    score, head = L.score_tokens(q, k, N=w.N, i0=w.i0, n=w.n, q_lo=0, q_hi=w.N, causal=True, want_head=True,
+                                 dev_status=flag)
+    torch.cuda.synchronize()
+    assert int(flag.item()) == 0
+    o_score, o_head = O.score_tokens(f64(q), f64(k), 0, w.N, w.i0, w.n, causal=True)
+    assert_scores_close(f64(score), o_score, what=f"{wname} all-rows score")
+    assert_scores_close(f64(head), o_head, what=f"{wname} all-rows score_head")
+    # every query row hands out probability 1 over the keys it sees: the per-head sums over ALL keys equal
+    # the number of rows, so the image share can never exceed it
+    assert float(score.sum(dim=1).max()) <= w.N + 1e-3
