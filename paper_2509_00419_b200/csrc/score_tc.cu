@@ -389,13 +389,19 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
     a.head_stride = d->head_stride ? d->head_stride : (int64_t)d->n;
     const size_t smem = 1024 + (size_t)kTileBytes * (1 + kStages) + sizeof(TcSmem);
     const int nqt = (Nq + kTile - 1) / kTile, nkt = (d->n + kTile - 1) / kTile;
-    // pass 2: when key tiles x KV heads do not fill the GPU, the query heads of a group are shared
-    // out over several CTAs (the smallest divisor of G that gets there, else all of G)
+    // pass 2: the query heads of a KV group can be shared out over hs CTAs (hs divides G).  More CTAs
+    // fill the GPU, fewer amortise a CTA's fixed cost over more tiles: take the hs with the smallest
+    // estimate waves x (fixed + tiles per CTA x per-tile), 296 CTAs to a wave (two per SM).
     int hsplit = 1;
-    for (int hs = 1; hs <= a.G; ++hs) {
-        if (a.G % hs) continue;
-        hsplit = hs;
-        if ((int64_t)nkt * d->Hkv * d->B * hs >= 148) break;
+    {
+        double best = 1e30;
+        for (int hs = 1; hs <= a.G; ++hs) {
+            if (a.G % hs) continue;
+            const int64_t ctas = (int64_t)nkt * d->Hkv * d->B * hs;
+            const double waves = (double)((ctas + 295) / 296);
+            const double est = waves * (5.0 + 0.6 * (a.G / hs) * nqt);
+            if (est < best - 1e-9) { best = est; hsplit = hs; }
+        }
     }
     a.hsplit = hsplit; a.nkt = nkt; a.ksplit = 1;
     if (lse) LVLM_RETURN_IF_CUDA(cudaMemsetAsync(cnt, 0, (size_t)d->B * nkt * 4, stream));
