@@ -410,3 +410,57 @@ def test_merge_nearest_kept(case):
         assert_rows_close(f64(Kd)[:, :, :M], want["Kc"], what="merged K rows")
         assert_rows_close(f64(Vd)[:, :, :M], want["Vc"], what="merged V rows")
         assert np.array_equal(f64(Kd)[:, :, i0 + k:M], f64(Kc)[:, :, i0 + n:])       # text rows only move
+
+
+# ------------------------------------------------------------------ library-internal cross-checks
+def test_score_tensor_core_kernel_agrees_with_cuda_core_kernel():
+    """Two independent CUDA implementations of the same scores (tcgen05 path, plain CUDA-core path)."""
+    r = np.random.default_rng(5)
+    B, N, i0, n, H, Hkv = 2, 700, 9, 600, 8, 2
+    Q = torch.from_numpy(r.normal(size=(B, N, H, 128)).astype(np.float32)).to(torch.bfloat16).cuda()
+    K = torch.from_numpy(r.normal(size=(B, Hkv, N, 128)).astype(np.float32)).to(torch.bfloat16).cuda()
+    lib = L.lib()
+    try:
+        lib.lvlm_debug_set_score_impl(1)
+        s_simt, h_simt = L.score_tokens(Q[:, 400:], K, N=N, i0=i0, n=n, q_lo=400, q_hi=N, want_head=True)
+        torch.cuda.synchronize()
+    finally:
+        lib.lvlm_debug_set_score_impl(0)
+    s_tc, h_tc = L.score_tokens(Q[:, 400:], K, N=N, i0=i0, n=n, q_lo=400, q_hi=N, want_head=True)
+    assert_scores_close(f64(s_tc), f64(s_simt), what="score, tensor-core vs CUDA-core")
+    assert_scores_close(f64(h_tc), f64(h_simt), what="score_head, tensor-core vs CUDA-core")
+
+
+def test_results_do_not_depend_on_programmatic_dependent_launch():
+    """The same chain of calls with and without programmatic dependent launch, bit for bit (no kernel
+    may touch its inputs before the kernels ahead of it have finished)."""
+    w = I.shrink(I.CFG1, n=448, T=64, C=512, planted=8)
+    lib = L.lib()
+
+    def chain():
+        hidden = I.hidden_states(w).cuda()
+        pos = torch.arange(w.N, dtype=torch.int32)[None].cuda()
+        Q, K, V = [t.cuda() for t in I.layer_qkv(w, 0, pos.cpu())]
+        k = w.n // 3
+        score, head = L.score_tokens(Q[:, w.n:], K, N=w.N, i0=0, n=w.n, q_lo=w.n, q_hi=w.N, want_head=True)
+        rank, _, _ = L.select_topk(score, k)
+        out, _ = L.merge_compact(hidden, rank, i0=0, k=k, Kc=K, Vc=V, pos_ids=pos)
+        M = out.shape[1]
+        ln = torch.full((w.B, w.Hkv), M, dtype=torch.int32, device="cuda")
+        acc = torch.rand(w.B, w.Hkv, w.N, device="cuda")
+        L.kv_compress(K, V, acc, ln, beta=0.9)
+        q = I.normal_bf16(w.seed, "pdl/q", (w.B, w.H, 128)).cuda()
+        dec = L.decode_attn(q, K, V, ln, acc_score=acc)
+        torch.cuda.synchronize()
+        return [score, rank, out, K, V, pos, ln, acc, dec]
+
+    try:
+        lib.lvlm_debug_set_pdl(0)
+        torch.manual_seed(3)
+        plain = chain()
+    finally:
+        lib.lvlm_debug_set_pdl(1)
+    torch.manual_seed(3)
+    overlapped = chain()
+    for a, b in zip(plain, overlapped):
+        assert torch.equal(a, b)
