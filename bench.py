@@ -374,6 +374,19 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
            "decode_frac_hbm": bytes_read / (t_dec * 1e6) / peaks["hbm_gbs"],
            "compress_us_per_layer": (t_cmp * 1e3 / (n_cmp * w.L)) if n_cmp else None,
            "final_len": cur_len, "launches": steps_total * w.L + n_cmp * 2}
+    # the same kernel with all layers folded into the batch of ONE call (not how a model decodes - its
+    # layers depend on each other - but it shows what the kernel streams when a launch is large)
+    nb = w.L * w.B
+    ws_f = L.alloc_workspace(L.OP_DECODE_ATTN, L.kv_dims(dec.K.view(nb, w.Hkv, w.cap, 128), H=w.H), device)
+    out_f = torch.empty(nb, w.H, 128, dtype=torch.bfloat16, device=device)
+    fold = lambda: L.decode_attn(qb.view(nb, w.H, 128), dec.K.view(nb, w.Hkv, w.cap, 128),
+                                 dec.V.view(nb, w.Hkv, w.cap, 128), dec.len.view(nb, w.Hkv),
+                                 acc_score=dec.acc.view(nb, w.Hkv, w.cap), out=out_f, ws=ws_f)
+    g_fold = P.capture(fold)
+    t_fold, _ = timed(g_fold.replay, 10, 3, flush)
+    by_fold = int(dec.len.sum().item()) * 128 * 2 * 2
+    res["folded_layers_one_call"] = {"ms": t_fold, "kv_bytes": by_fold, "gbs": by_fold / (t_fold * 1e6),
+                                     "frac_hbm": by_fold / (t_fold * 1e6) / peaks["hbm_gbs"]}
     if n_cmp:
         # bytes a compression has to move: every moved row of K and V read and written once, all scores
         # read (counted on the first compression; the later ones evict the same number of entries)
