@@ -89,6 +89,8 @@ typedef struct lvlm_dims {
     int32_t causal;   /* scoring: 1 = row at position p sees keys j <= p; 0 = sees all N keys */
     int32_t recent;   /* kv_compress: this many newest entries of every head are never evicted */
     int32_t merge_mode; /* lvlm_workspace_bytes(LVLM_OP_MERGE_COMPACT): the lvlm_merge_mode to size for */
+    int32_t cache_stable; /* decode_attn: 1 = Kc, Vc and len are neither written nor still being read by the
+                             operation enqueued just before this call (see lvlm_decode_attn) */
     int64_t q_stride_b, q_stride_n, q_stride_h;  /* Q[b][i][h][D]; default packed [B][q_hi-q_lo][H][D] */
     int64_t kv_stride_b, kv_stride_h;            /* K,V[b][g][row][D], rows packed; default [B][Hkv][cap][D] */
     int64_t hid_stride_b;                        /* hidden[b][row][C], rows packed; default N*C */
@@ -217,6 +219,11 @@ lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, int32_t* pos,
  * A head with len == 0 (and no append) outputs zeros.  A head whose len lies outside [0, cap]
  * is skipped: zeros are written, nothing is appended, its len is left alone and
  * LVLM_DEV_BOUNDS is set.
+ * d->cache_stable = 1 promises that the operation enqueued on the stream just before this call
+ * does not write Kc, Vc or len (true between the layers of a model: the cache of a layer was last
+ * written in the previous decoding step; NOT true right after lvlm_kv_compress or
+ * lvlm_merge_compact on the same cache).  The kernel then starts fetching the cache while that
+ * operation is still draining; q, k_new, v_new and all writes wait for it as always.
  * Workspace: only used when acc_score is given (the scaled logits are parked there between
  * the pass over the keys and the update of acc_score); its contents need not be zeroed.
  * Reads d: B,H,Hkv,D,cap,kv_stride_*.

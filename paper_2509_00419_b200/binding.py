@@ -31,7 +31,7 @@ class Dims(ctypes.Structure):
     """Mirror of ``lvlm_dims``."""
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "H", "Hkv", "D", "N", "C", "cap", "i0", "n", "k", "q_lo", "q_hi", "causal",
-                 "recent", "merge_mode")] + \
+                 "recent", "merge_mode", "cache_stable")] + \
                [(n, ctypes.c_int64) for n in
                 ("q_stride_b", "q_stride_n", "q_stride_h", "kv_stride_b", "kv_stride_h",
                  "hid_stride_b", "out_stride_b", "head_stride")]
@@ -247,11 +247,12 @@ def kv_compress(Kc, Vc, acc_score, length, *, beta=1.0, budget=0, recent=0, e_lo
 
 
 def decode_attn(q, Kc, Vc, length, *, k_new=None, v_new=None, acc_score=None, scale=None, out=None,
-                ws=None, dev_status=None, stream=None):
+                ws=None, dev_status=None, stream=None, cache_stable=False):
     """lvlm_decode_attn.  q [B,H,D]; returns out [B,H,D] bf16.  Kc, Vc, length and acc_score are
     updated in place when k_new/v_new or acc_score are given."""
     B, H, D = q.shape
     d = kv_dims(Kc, H=H)
+    d.cache_stable = int(bool(cache_stable))
     if scale is None:
         scale = 1.0 / math.sqrt(D)
     if out is None:

@@ -117,6 +117,7 @@ struct DecodeArgs {
     const __nv_bfloat16* q; __nv_bfloat16* Kc; __nv_bfloat16* Vc; int32_t* len;
     const __nv_bfloat16* k_new; const __nv_bfloat16* v_new; float* acc_score; __nv_bfloat16* out;
     int H, Hkv, cap, S;
+    int early;               // the cache and len are not written by the kernel ahead: fetch before waiting for it
     int64_t kv_sb, kv_sh;
     float scale_log2;
     float* ws_s;             // [B*H][cap] scaled logits (log2 domain), only with acc_score
@@ -137,7 +138,9 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
     float* s_rm = s_FI + 8;                                             // [S][8] max of every CTA of the cluster
     float* s_rl = s_rm + 8 * kDecMaxCluster;                            // [S][8] sum of every CTA
 
-    pdl_enter();
+    // With a.early the first key/value tiles and the length are fetched while the kernel ahead in the
+    // stream is still finishing; q, k_new, v_new and every write come after the wait in any case.
+    if (!a.early) pdl_enter();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.S, H = a.H, cap = a.cap;
     const int hd = blockIdx.x / S;
@@ -153,6 +156,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
         atomicOr(a.dev_status, LVLM_DEV_BOUNDS);                        // bad length, or append at capacity
     const int lne = ln + (app ? 1 : 0);
     if (lne == 0) {                                                     // no key at all: zeros
+        if (a.early) pdl_enter();
         if (rank == 0)
             for (int i = tid; i < G * kHeadDim; i += kDecThreads)
                 a.out[(int64_t)(b * H + h0) * kHeadDim + i] = __float2bfloat16_rn(0.f);
@@ -186,20 +190,11 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
             const int e = u * 32 + lane;
             const int r = e >> 4, ch = e & 15;
             const int j = j0 + r;
-            const bool ok = j < lne;
-            const bool fresh = app && j == ln;
-            const __nv_bfloat16* ksrc = fresh ? kn : Kseq + (int64_t)(ok ? j : 0) * kHeadDim;
-            const __nv_bfloat16* vsrc = fresh ? vn : Vseq + (int64_t)(ok ? j : 0) * kHeadDim;
+            const bool ok = j < ln;            // rows the cache already holds; an appended row is put in place later
+            const int64_t ro = (int64_t)(ok ? j : 0) * kHeadDim + ch * 8;
             const uint32_t off = r * 256 + ((ch ^ (r & 7)) << 4);
-            cp_async16_zfill(st + off, ksrc + ch * 8, ok ? 16 : 0);
-            cp_async16_zfill(st + kTileHalf + off, vsrc + ch * 8, ok ? 16 : 0);
-        }
-        // the warp that meets the appended row also stores it into the cache
-        if (app && ln >= j0 && ln < j0 + kTileKeys) {
-            const uint2 kv = reinterpret_cast<const uint2*>(kn)[lane];
-            const uint2 vv = reinterpret_cast<const uint2*>(vn)[lane];
-            reinterpret_cast<uint2*>(Kseq + (int64_t)ln * kHeadDim)[lane] = kv;
-            reinterpret_cast<uint2*>(Vseq + (int64_t)ln * kHeadDim)[lane] = vv;
+            cp_async16_zfill(st + off, Kseq + ro, ok ? 16 : 0);
+            cp_async16_zfill(st + kTileHalf + off, Vseq + ro, ok ? 16 : 0);
         }
     };
 #pragma unroll
@@ -208,6 +203,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
         cp_async_commit();
     }
 
+    if (a.early) pdl_enter();
     // query fragments: heads of the group are rows 0..G-1 of a 16-row A tile
     uint32_t qa[8][2];
 #pragma unroll
@@ -229,6 +225,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
         __syncwarp();
         const uint32_t st = ring + (it % kStagesDec) * kStageBytes;
         const int j0 = (t_lo + warp + it * kDecWarps) * kTileKeys;
+        if (app && ln >= j0 && ln < j0 + kTileKeys) {
+            // the appended row: into its place of the tile (zero-filled by the copy) and into the cache
+            const int rr = ln - j0, ch = lane & 15;
+            const uint4 x = *reinterpret_cast<const uint4*>((lane < 16 ? kn : vn) + ch * 8);
+            const uint32_t off = (lane < 16 ? 0 : kTileHalf) + rr * 256 + ((ch ^ (rr & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st + off), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
+            *reinterpret_cast<uint4*>((lane < 16 ? Kseq : Vseq) + (int64_t)ln * kHeadDim + ch * 8) = x;
+            __syncwarp();
+        }
         // ---- S = Q K^T for 16 keys -------------------------------------------------------------------
         float s[2][4];
 #pragma unroll
@@ -466,6 +471,7 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
     a.acc_score = acc_score;
     a.out = static_cast<__nv_bfloat16*>(out);
     a.H = d->H; a.Hkv = d->Hkv; a.cap = d->cap; a.S = L.S;
+    a.early = d->cache_stable != 0 && pdl_enabled();
     a.kv_sb = kv_sb; a.kv_sh = kv_sh; a.scale_log2 = scale * kLog2e;
     a.ws_s = acc_score ? reinterpret_cast<float*>(wsb + L.off_s) : nullptr;
     a.dev_status = dev_status;

@@ -150,13 +150,15 @@ class DecodeLayers:
         self.ws_kv = L.alloc_workspace(L.OP_KV_COMPRESS, dk, device)
 
     def decode_step(self, q, k_new=None, v_new=None, accumulate=True, layers=None):
-        """q [layer][B][H][D]; k_new, v_new [layer][B][Hkv][D] or None."""
-        for l in (range(self.nl) if layers is None else layers):
+        """q [layer][B][H][D]; k_new, v_new [layer][B][Hkv][D] or None.  The first layer of a step may
+        follow a compression of its own cache; every other layer follows the decode call of another
+        layer, which does not touch this layer's cache, so its fetches may start early."""
+        for i, l in enumerate(range(self.nl) if layers is None else layers):
             L.decode_attn(q[l], self.K[l], self.V[l], self.len[l],
                           k_new=None if k_new is None else k_new[l],
                           v_new=None if v_new is None else v_new[l],
                           acc_score=self.acc[l] if (accumulate and self.acc is not None) else None,
-                          out=self.out[l], ws=self.ws_dec, dev_status=self.status)
+                          out=self.out[l], ws=self.ws_dec, dev_status=self.status, cache_stable=i > 0)
 
     def compress(self, beta=1.0, budget=0, recent=0, e_lo=None, e_hi=None, first_layer=0):
         nl = self.nl - first_layer
