@@ -24,13 +24,13 @@ constexpr int kNoRow = -2147483647 - 1;  // marks a slot of the four-row group t
 constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
 
 // One wave of CTAs over the whole batch (four per SM fit for rows up to 4096 channels, two beyond:
-// the registers of the row groups in flight decide), at least 32 input rows each (few partial sums to add at the end); clusters of 8.
+// the registers of the row groups in flight decide), at least 8 input rows each; clusters of 8.
 HiddenGrid hidden_grid(const lvlm_dims* d) {
     HiddenGrid g;
     g.V = d->C / 8;
     const int per_sm = (g.V + kHidThreads - 1) / kHidThreads <= 2 ? 4 : 2;
     int cps = (per_sm * 148) / d->B;
-    const int max_by_rows = (d->N + 31) / 32;
+    const int max_by_rows = (d->N + 7) / 8;
     cps = cps > max_by_rows ? max_by_rows : cps;
     cps = cps < 1 ? 1 : cps;
     g.cl = cps >= kHidCluster ? kHidCluster : 1;
