@@ -151,7 +151,7 @@ def bench_prefill(w, device, steps, warmup, flush, peaks, breakdown=True):
                 "merge_compact_frac_hbm": by / (t_me * 1e6) / peaks["hbm_gbs"],
                 "score_tflops": st.flops_score() / (t_sc * 1e9),
                 "score_frac_tensor": st.flops_score() / (t_sc * 1e9) / peaks["bf16_tflops"]})
-        # the spec merge variant on stage 1: every dropped token into its most similar kept token
+        # the similarity-merge variant (not in the paper) on stage 1: every dropped token into its most similar kept token
         from paper_2509_00419_b200 import binding as L
         st0 = run.stages[0]
         nk = P.ReduceStage(st0.B, st0.N, st0.C, st0.H, st0.Hkv, st0.cap, st0.i0, st0.n, st0.M, device,

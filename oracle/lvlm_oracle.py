@@ -14,7 +14,7 @@ Section 3.2.2 KV-cache compression, Appendix A.2 settings):
   select_topk     split into P_unmerged / P_merged by A, ordered   Sec. 3.2.1 par. 4
   merge_weights   the weight list W_v                              Sec. 3.2.1 par. 4
   merge_compact   P_new = W_v x P_merged; P_compressed             Sec. 3.2.1 par. 4
-  nearest_kept_merge  the spec variant (no paper passage)    --
+  nearest_kept_merge  similarity-merge variant (no paper passage)   --
   kv_compress     sort A, keep prefix reaching beta, drop the rest Sec. 3.2.2 par. 2
   decode_attn     current token attends to every cached K, V       Sec. 3.2.2 par. 1
   pyramid_schedule constant reduction ratio from the final budget  App. A.2
@@ -243,7 +243,7 @@ def merge_compact(hidden, rank, i0, n, k, mode=LINEAR_RANK, custom=None,
 
 
 def nearest_kept_merge(hidden, rank, i0, n, k, mass=None, Kc=None, Vc=None, pos_ids=None, assign=None):
-    """North-star variant (not in the paper): every dropped image token is merged into
+    """Similarity-merge variant (not in the paper): every dropped image token is merged into
     the kept image token it is most similar to.
 
     For a dropped token d (rank >= k): a(d) = argmax over kept t of the cosine

@@ -349,7 +349,7 @@ def test_cfg1_pipeline():
     assert_scores_close(ad.cpu().numpy()[:, :, :m], o_dec["acc_score"][:, :, :m], what="cfg1 acc")
 
 
-# ------------------------------------------------------------------ nearest-kept merge (spec variant)
+# ------------------------------------------------------------------ nearest-kept merge (variant that is not in the paper)
 NK_CASES = [  # B, N, i0, n, C, k, Hkv, with_mass, with_kv
     (1, 40, 3, 30, 64, 7, 1, False, False), (2, 700, 5, 640, 256, 300, 2, True, True),
     (1, 1500, 0, 1400, 200, 130, 2, False, True), (3, 333, 2, 300, 1024, 299, 1, True, False),
