@@ -528,7 +528,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="lvlm", choices=["lvlm", "reference"])
-    ap.add_argument("--extras", default="cfg1,cfg3,cfg4,cfg5")
+    ap.add_argument("--extras", default="cfg1,cfg3,cfg4,cfg5,video")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode loop length")
     ap.add_argument("--only", default="", choices=["", "step", "prefill", "decode"],
                     help="run one piece and print its JSON: 'step' = the timed headline loop alone "
@@ -675,6 +675,20 @@ def main():
             except Exception as e:          # an extra must not take the headline down
                 import traceback
                 extras[name] = {"error": repr(e), "trace": traceback.format_exc()[-600:]}
+        # how many image entries per head the cumulative-attention threshold keeps, by beta (Section 3.2.2:
+        # shallow layers keep more, deep layers fewer; here every layer has the same synthetic mass profile)
+        sweep = {}
+        for beta in (0.9, 0.95, 0.99, 0.995, 0.999):
+            fp.restore()
+            fp.phase_score_caches()
+            fp.dec.compress(beta=beta, e_lo=fp.e_lo, e_hi=fp.e_hi, first_layer=fp.first)
+            torch.cuda.synchronize()
+            img_before = torch.tensor([fp.lens[l] - w.T - w.i0 for l in range(fp.first, w.L)], device=device).float()
+            kept = fp.dec.len[fp.first:].float().mean(dim=(1, 2)) - w.T - w.i0
+            sweep[str(beta)] = {"mean_kept_image_entries": float(kept.mean().item()),
+                                "mean_kept_fraction": float((kept / img_before).mean().item())}
+        fp.restore()
+        extras["beta_sweep_" + w.name] = sweep
         out["workloads"] = extras
         out["cpu_baseline"] = cpu_baseline(w)
     elif rank == 0:

@@ -541,7 +541,7 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
     NkLayout L;
     if (!nk_layout(d, &L) || d->k < 1) return LVLM_ERR_INVALID_ARG;
     if (!hidden_out || hidden_out == hidden) return LVLM_ERR_UNSUPPORTED;     // out of place only
-    if (L.r > kMaxSortN) return LVLM_ERR_UNSUPPORTED;          // one slice of the keys has to fit in shared memory
+    if (L.r > kRankMaxKeys) return LVLM_ERR_UNSUPPORTED;       // the slices of the keys have to fit in shared memory
     if (!ws || !aligned256(ws) || ws_bytes < L.total) return LVLM_ERR_WORKSPACE;
     const int64_t hid_sb = d->hid_stride_b ? d->hid_stride_b : (int64_t)d->N * d->C;
     const int64_t out_sb = d->out_stride_b ? d->out_stride_b : (int64_t)L.Nout * d->C;

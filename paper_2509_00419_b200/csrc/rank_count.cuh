@@ -10,6 +10,8 @@ namespace lvlm {
 
 constexpr int kRankThreads = 256;
 constexpr int kRankMaxCluster = 8;
+constexpr int kRankMaxSlice = 16384;       // keys of one slice in shared memory (128 KB)
+constexpr int kRankMaxKeys = kRankMaxCluster * kRankMaxSlice;     // 131072 keys per sequence
 
 __device__ __forceinline__ uint32_t rank_cluster_rank() {
     uint32_t r;
@@ -34,6 +36,7 @@ inline void rank_shape(int n, int B, int* S, int* slice_len) {
     const int jblocks = (n + kRankThreads - 1) / kRankThreads;
     int s = 1;
     while (s < kRankMaxCluster && (int64_t)jblocks * B * (2 * s) <= 8 * 148 && n / (2 * s) >= 256) s *= 2;
+    while (s < kRankMaxCluster && (n + s - 1) / s > kRankMaxSlice) s *= 2;       // a slice has to fit
     *S = s;
     *slice_len = (((n + s - 1) / s) + 1) & ~1;
 }

@@ -89,7 +89,7 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
     if (!score || !rank || B <= 0 || n <= 0 || k < 0 || k > n) return LVLM_ERR_INVALID_ARG;
     if (score_stride == 0) score_stride = n;
     if (score_stride < n) return LVLM_ERR_INVALID_ARG;
-    if (n > kMaxSortN) return LVLM_ERR_UNSUPPORTED;
+    if (n > kRankMaxKeys) return LVLM_ERR_UNSUPPORTED;
     int S, slice_len;
     rank_shape(n, B, &S, &slice_len);
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_count_kernel,

@@ -181,7 +181,13 @@ CFG5 = Workload("cfg5", seed=5, B=1, L=48, C=6144, H=48, Hkv=8, n=16384, T=256,
                 stages=((2, 4096), (12, 492)), planted=128, centroids=1024,
                 decode_steps=2048, budget=512, trigger=128, recent=128, cap=768, beta=1.0)
 
-WORKLOADS = {w.name: w for w in (CFG1, CFG2, CFG2_ALT, CFG3, CFG4, CFG5)}
+# A video-length prompt (Section 4.2 evaluates video benchmarks with the same keep ratios): 64 frames of
+# 512 tokens on the 7B-class shapes, 15 % kept after three stages at a constant ratio (32768 -> 17411
+# -> 9251 -> 4915).
+VIDEO = Workload("video", seed=7, B=1, L=28, C=3584, H=28, Hkv=4, n=32768, T=128,
+                 stages=((5, 17411), (9, 9251), (13, 4915)), planted=256, centroids=1024, decode_steps=1)
+
+WORKLOADS = {w.name: w for w in (CFG1, CFG2, CFG2_ALT, CFG3, CFG4, CFG5, VIDEO)}
 
 
 def shrink(w: Workload, **kw) -> Workload:

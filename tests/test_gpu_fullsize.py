@@ -87,6 +87,11 @@ def test_cfg5_extreme_reduction_full_size():
     _check_pyramid(I.CFG5, sample=[0])
 
 
+def test_video_length_pyramid_full_size():
+    """32768 image tokens (64 frames): the second workload shape the paper evaluates (video benchmarks)."""
+    _check_pyramid(I.VIDEO, sample=[0])
+
+
 def _decode_chunks(w, n_layers, prompt_len, steps, check_steps, dev):
     """Decode loop with the periodic budgeted compression at the workload's full batch and head
     counts, on ``n_layers`` layers.  The oracle restarts from a copy of the GPU state at the start of
