@@ -171,7 +171,8 @@ lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_str
  *   new_len     optional [B] int32 out: rows after the call
  * Reads d: B,N,C,Hkv,D,cap,i0,n,k,hid_stride_b,out_stride_b,kv_stride_*.
  * Errors: INVALID_ARG (NULL hidden/rank, i0+n>N, k outside [0,n], N>cap with Kc, only one of
- * Kc/Vc, CUSTOM without w_custom, C%8), UNSUPPORTED (D!=128 with Kc), ALIGNMENT, WORKSPACE.
+ * Kc/Vc, CUSTOM without w_custom, C%8), UNSUPPORTED (D!=128 with Kc; C > 8192 with hidden_out;
+ * NEAREST_KEPT without hidden_out), ALIGNMENT, WORKSPACE.
  */
 lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* Kc, void* Vc,
                                int32_t* pos_ids, const int32_t* rank, const lvlm_dims* d,
