@@ -266,12 +266,19 @@ class FullPass:
         return self.pre.launches + 2 * len(self.groups) + 2 + w.L
 
 
-def bench_full(w, device, steps, warmup, flush, peaks, phases=True):
+def bench_full(w, device, steps, warmup, flush, peaks, phases=True, fence=None):
+    """``fence`` (a barrier over the ranks plus a device synchronise) brackets the timed steps."""
     from paper_2509_00419_b200 import pipeline as P
     fp = FullPass(w, device)
     g = P.capture(fp.step)
     fp.restore()
-    ms, per_step = timed(g.replay, steps, warmup, flush, between=fp.restore)
+    for _ in range(warmup):                   # warm-up steps, then the ranks line up
+        fp.restore(); flush(); g.replay()
+    if fence is not None:
+        fence()
+    ms, per_step = timed(g.replay, steps, 0, flush, between=fp.restore)
+    if fence is not None:
+        fence()
     if not phases:
         return {"ms_per_step": ms, "launches": fp.launches, "tokens_in": fp.pre.tokens_in}, fp, per_step
     # phases, timed one by one (each from the restored state it expects)
@@ -581,8 +588,13 @@ def main():
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
+    def fence():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
     res, fp, per_step = bench_full(w, device, args.steps, args.warmup, flush, peaks,
-                                   phases=args.only != "step")
+                                   phases=args.only != "step", fence=fence)
     torch.cuda.synchronize()
     clocks = sampler.stop()
     if args.only == "step":
