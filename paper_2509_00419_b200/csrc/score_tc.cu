@@ -75,14 +75,26 @@ __device__ __forceinline__ float ex2_fast(float x) {
 // Pass 1, one chunk of 32 raw logits of a query row: columns [0, lim) are visible.  Updates the running
 // (max, sum of 2^(logit*scale - max)).  Four partial sums keep the adds off one dependency chain.
 __device__ __forceinline__ void rowstat_chunk(float* v, int lim, float scale_log2, float& m_run, float& l_run) {
-    float cmax = -INFINITY;
-    if (lim >= 32) {
+    if (lim >= 32 && scale_log2 > 0.f) {
+        // every column visible: the maximum is taken on the raw logits (a positive scale keeps the order)
+        // and the scale is folded into the exponent's multiply-add
+        float cmax = v[0];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) { v[c] *= scale_log2; cmax = fmaxf(cmax, v[c]); }
-    } else {
+        for (int c = 1; c < 32; ++c) cmax = fmaxf(cmax, v[c]);
+        const float m_new = fmaxf(m_run, cmax * scale_log2);
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) { v[c] = c < lim ? v[c] * scale_log2 : -INFINITY; cmax = fmaxf(cmax, v[c]); }
+        for (int c = 0; c < 32; c += 4) {
+            s0 += ex2_fast(fmaf(v[c], scale_log2, -m_new)); s1 += ex2_fast(fmaf(v[c + 1], scale_log2, -m_new));
+            s2 += ex2_fast(fmaf(v[c + 2], scale_log2, -m_new)); s3 += ex2_fast(fmaf(v[c + 3], scale_log2, -m_new));
+        }
+        l_run = l_run * ex2_fast(m_run - m_new) + ((s0 + s1) + (s2 + s3));
+        m_run = m_new;
+        return;
     }
+    float cmax = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) { v[c] = c < lim ? v[c] * scale_log2 : -INFINITY; cmax = fmaxf(cmax, v[c]); }
     const float m_new = fmaxf(m_run, cmax);
     if (m_new > -INFINITY) {
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
