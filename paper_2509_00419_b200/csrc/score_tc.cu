@@ -280,6 +280,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
 #pragma unroll 1
             for (int c2 = 0; c2 < 2; ++c2) {
                 const int c4 = half * 2 + c2;                  // 32-column chunk of the tile
+                // nothing to do where the tile sticks out of the window: a warp whose 32 query rows lie past
+                // it (pass 1), a chunk whose 32 query rows lie past it (pass 2)
+                if (MODE == 0 && qt * kTile + quarter * 32 >= a.Nq) continue;
+                if (MODE == 1 && q2 * kTile + c4 * 32 >= a.Nq) continue;
                 float v[32];
                 tmem_ld32(lane_addr + buf * kTile + c4 * 32, v);
                 tmem_ld_wait();
