@@ -3,12 +3,12 @@
 // somebody else still has to read.
 //
 // A sequence (or, for wide rows, one group of its columns: column groups never interact) is
-// walked by one thread-block cluster in super-tiles of S x R consecutive output positions, CTA
-// `rank` owning R of them.  Per super-tile every CTA stages the source rows of its positions in
-// shared memory (cp.async), adds the merged (dropped) rows that sit in its position range to fp32
-// accumulators, and only after a cluster barrier - when every CTA has its sources on chip -
-// overwrites its positions.  The sources of the next super-tile lie beyond everything written so
-// far, so they are fetched into a second buffer while the current one is being stored.
+// walked by one thread-block cluster in super-tiles of S x R consecutive positions, CTA `rank`
+// owning R of them.  Per super-tile every CTA stages rows in shared memory (cp.async) - the source
+// rows of its output positions, or, when rows are merged, its input rows themselves - and only after
+// a cluster barrier, when every CTA has its rows on chip, writes: a row goes to its destination,
+// a merged row is added to fp32 sums.  What the next super-tile needs lies beyond everything written
+// so far, so it is fetched into a second buffer while the current one is being stored.
 // With many independent sequences S is 1 and the barrier is a block barrier.
 #include "compact.cuh"
 
@@ -25,7 +25,7 @@ struct InplaceArgs {
     int64_t stride_b, stride_g;
     int G, V, Vsub, S, Nout, N, n, i0, merged_row, meta_stride, maps_per_g, Rmax, CG, RL;
     int64_t map_stride;
-    const int32_t* src_map; const float* wgt; const int32_t* meta; const int32_t* nout;
+    const int32_t* src_map; const int32_t* dst_map; const float* wgt; const int32_t* meta; const int32_t* nout;
 };
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
@@ -81,9 +81,16 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
     R = min(R, a.Rmax);
     const int Rc = R * S;
     uint4* buf[2] = {tile, tile + (size_t)a.Rmax * a.Vsub};
-    // source row of each of my positions, three super-tiles deep: fetched two rounds ahead so
-    // that no copy ever waits for its index
+    // Two ways to walk a sequence.  Without merged rows (w == NULL) the walk is over OUTPUT positions: a
+    // position's source row is staged (rows that are dropped are never read).  With merged rows the walk is
+    // over INPUT positions: every row from the first change on is staged exactly once, in order, and then
+    // either stored to its destination (at or before it) or added, times its weight, to the sums.
+    // Per position of a super-tile: s_idx = row to copy from / to (-1: nothing, -2: merged row), s_wt = weight;
+    // both are fetched two rounds ahead so that no copy ever waits for them.
+    const bool by_input = w != nullptr;
+    const int32_t* dst = by_input ? a.dst_map + (int64_t)b * a.map_stride : nullptr;
     int32_t* s_idx = reinterpret_cast<int32_t*>(tile + 2 * (size_t)a.Rmax * a.Vsub);     // [3][Rmax]
+    float* s_wt = reinterpret_cast<float*>(s_idx + 3 * a.Rmax);                          // [3][Rmax]
     constexpr int kIdxPerThread = 2;                     // Rmax <= 2 * blockDim.x
 
     float acc[MAXC][8];
@@ -92,32 +99,43 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
 
-    // -1: nothing to copy (beyond the end, the merged row, or a row that stays where it is)
-    auto fetch_idx = [&](int t0, int* reg) {
+    auto fetch_idx = [&](int t0, int* reg, float* regw) {
 #pragma unroll
         for (int u = 0; u < kIdxPerThread; ++u) {
             const int rr = threadIdx.x + u * kCompactThreads;
             const int o = t0 + rank * R + rr;
-            int sidx = -1;
-            if (rr < R && o < Nout) { sidx = src[o]; if (sidx == o) sidx = -1; }
-            reg[u] = sidx;
+            int v = -1;
+            float wv = 0.f;
+            if (rr < R) {
+                if (!by_input) {
+                    if (o < Nout) { v = src[o]; if (v == o) v = -1; }
+                } else if (o < a.N) {
+                    const int d = dst[o];                                  // two independent loads
+                    wv = (o >= a.i0 && o < a.i0 + a.n) ? w[o - a.i0] : 0.f;
+                    if (d >= 0) { v = d == o ? -1 : d; wv = 0.f; }
+                    else v = wv != 0.f ? -2 : -1;
+                }
+            }
+            reg[u] = v;
+            regw[u] = wv;
         }
     };
-    auto put_idx = [&](int slot, const int* reg) {
+    auto put_idx = [&](int slot, const int* reg, const float* regw) {
 #pragma unroll
         for (int u = 0; u < kIdxPerThread; ++u) {
             const int rr = threadIdx.x + u * kCompactThreads;
-            if (rr < R) s_idx[slot * a.Rmax + rr] = reg[u];
+            if (rr < R) { s_idx[slot * a.Rmax + rr] = reg[u]; s_wt[slot * a.Rmax + rr] = regw[u]; }
         }
     };
-    auto load_tile = [&](int slot, uint4* dst) {
+    auto load_tile = [&](int t0, int slot, uint4* dstbuf) {
         for (int rr = rl; rr < R; rr += RL) {
-            const int sidx = s_idx[slot * a.Rmax + rr];
-            if (sidx >= 0) {
+            const int v = s_idx[slot * a.Rmax + rr];
+            if (v != -1) {
+                const int64_t from = by_input ? (int64_t)(t0 + rank * R + rr) : (int64_t)v;
 #pragma unroll
                 for (int ci = 0; ci < MAXC; ++ci) {
                     const int c = cg + ci * CG;
-                    if (c < vw) cp_async16(&dst[rr * a.Vsub + c], rows + (int64_t)sidx * V + c);
+                    if (c < vw) cp_async16(&dstbuf[rr * a.Vsub + c], rows + from * V + c);
                 }
             }
         }
@@ -126,80 +144,51 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
 
     {
         int reg[kIdxPerThread];
-        fetch_idx(o_start, reg);
-        put_idx(0, reg);
-        fetch_idx(o_start + Rc, reg);
-        put_idx(1, reg);
+        float regw[kIdxPerThread];
+        fetch_idx(o_start, reg, regw);
+        put_idx(0, reg, regw);
+        fetch_idx(o_start + Rc, reg, regw);
+        put_idx(1, reg, regw);
         __syncthreads();
     }
-    load_tile(0, buf[0]);
+    load_tile(o_start, 0, buf[0]);
     int k = 0;
     for (int t0 = o_start; t0 < Nscan; t0 += Rc, ++k) {
-        if (t0 + Rc < Nscan) load_tile((k + 1) % 3, buf[(k + 1) & 1]);
+        if (t0 + Rc < Nscan) load_tile(t0 + Rc, (k + 1) % 3, buf[(k + 1) & 1]);
         else cp_async_commit_group();
         int reg[kIdxPerThread];
-        fetch_idx(t0 + 2 * Rc, reg);                  // in flight while this round runs
-        if (w) {
-            // merged rows inside my positions: read before anyone overwrites them; kWB rows in flight
-            constexpr int kWB = 4;
-            for (int rb = rl; rb < R; rb += kWB * RL) {
-                float wj[kWB];
-                uint4 x[kWB][MAXC];
-#pragma unroll
-                for (int u = 0; u < kWB; ++u) {
-                    const int rr = rb + u * RL;
-                    const int o = t0 + rank * R + rr;
-                    wj[u] = (rr < R && o < Nscan && o >= a.i0 && o < a.i0 + a.n) ? w[o - a.i0] : 0.f;
-                }
-#pragma unroll
-                for (int u = 0; u < kWB; ++u) {
-                    const int o = t0 + rank * R + rb + u * RL;
-#pragma unroll
-                    for (int ci = 0; ci < MAXC; ++ci) {
-                        const int c = cg + ci * CG;
-                        x[u][ci] = (wj[u] != 0.f && c < vw) ? rows[(int64_t)o * V + c] : make_uint4(0, 0, 0, 0);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < kWB; ++u) {
-                    if (wj[u] != 0.f) {
-#pragma unroll
-                        for (int ci = 0; ci < MAXC; ++ci) {
-                            const uint4 xv = x[u][ci];
-                            acc[ci][0] = fmaf(wj[u], bf16_lo(xv.x), acc[ci][0]); acc[ci][1] = fmaf(wj[u], bf16_hi(xv.x), acc[ci][1]);
-                            acc[ci][2] = fmaf(wj[u], bf16_lo(xv.y), acc[ci][2]); acc[ci][3] = fmaf(wj[u], bf16_hi(xv.y), acc[ci][3]);
-                            acc[ci][4] = fmaf(wj[u], bf16_lo(xv.z), acc[ci][4]); acc[ci][5] = fmaf(wj[u], bf16_hi(xv.z), acc[ci][5]);
-                            acc[ci][6] = fmaf(wj[u], bf16_lo(xv.w), acc[ci][6]); acc[ci][7] = fmaf(wj[u], bf16_hi(xv.w), acc[ci][7]);
-                        }
-                    }
-                }
-            }
-        }
-        if (w && t0 + Rc < Nscan) {
-            // the merged rows of the next round's positions start their way from DRAM now (L2 prefetch,
-            // one request per 128 bytes); nothing overwrites them before that round
-            const int lines = (vw * 16 + 127) / 128;
-            for (int e = threadIdx.x; e < R * lines; e += kCompactThreads) {
-                const int o = t0 + Rc + rank * R + e / lines;
-                if (o < Nscan && o >= a.i0 && o < a.i0 + a.n)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(rows + (int64_t)o * V + (e % lines) * 8));
-            }
-        }
-        cp_async_wait_group<1>();                     // this super-tile's sources have landed
+        float regw[kIdxPerThread];
+        fetch_idx(t0 + 2 * Rc, reg, regw);            // in flight while this round runs
+        cp_async_wait_group<1>();                     // this super-tile's rows have landed
         cluster_barrier();                            // ... in every CTA of the cluster
         const uint4* cur = buf[k & 1];
         const int32_t* cur_idx = s_idx + (k % 3) * a.Rmax;
+        const float* cur_wt = s_wt + (k % 3) * a.Rmax;
         for (int rr = rl; rr < R; rr += RL) {
-            if (cur_idx[rr] >= 0) {
-                const int o = t0 + rank * R + rr;
+            const int v = cur_idx[rr];
+            if (v >= 0) {
+                const int64_t to = by_input ? (int64_t)v : (int64_t)(t0 + rank * R + rr);
 #pragma unroll
                 for (int ci = 0; ci < MAXC; ++ci) {
                     const int c = cg + ci * CG;
-                    if (c < vw) rows[(int64_t)o * V + c] = cur[rr * a.Vsub + c];
+                    if (c < vw) rows[to * V + c] = cur[rr * a.Vsub + c];
+                }
+            } else if (v == -2) {
+                const float wj = cur_wt[rr];
+#pragma unroll
+                for (int ci = 0; ci < MAXC; ++ci) {
+                    const int c = cg + ci * CG;
+                    if (c < vw) {
+                        const uint4 xv = cur[rr * a.Vsub + c];
+                        acc[ci][0] = fmaf(wj, bf16_lo(xv.x), acc[ci][0]); acc[ci][1] = fmaf(wj, bf16_hi(xv.x), acc[ci][1]);
+                        acc[ci][2] = fmaf(wj, bf16_lo(xv.y), acc[ci][2]); acc[ci][3] = fmaf(wj, bf16_hi(xv.y), acc[ci][3]);
+                        acc[ci][4] = fmaf(wj, bf16_lo(xv.z), acc[ci][4]); acc[ci][5] = fmaf(wj, bf16_hi(xv.z), acc[ci][5]);
+                        acc[ci][6] = fmaf(wj, bf16_lo(xv.w), acc[ci][6]); acc[ci][7] = fmaf(wj, bf16_hi(xv.w), acc[ci][7]);
+                    }
                 }
             }
         }
-        put_idx((k + 2) % 3, reg);
+        put_idx((k + 2) % 3, reg, regw);
         __syncthreads();                              // buffer and index slot are reused in the next round
     }
     cp_async_wait_group<0>();
@@ -241,8 +230,11 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
                                    int B, int G, int V, int Nout, const int32_t* src_map,
                                    const float* wgt, const int32_t* meta, int N, int n, int i0,
                                    int merged_row, int meta_stride, cudaStream_t stream,
-                                   int maps_per_g, int64_t map_stride, const int32_t* nout) {
+                                   int maps_per_g, int64_t map_stride, const int32_t* nout,
+                                   const int32_t* dst_map) {
     InplaceArgs a;
+    if (wgt && !dst_map) return LVLM_ERR_INVALID_ARG;      // merged rows need the destination map
+    a.dst_map = dst_map;
     a.base0 = static_cast<char*>(base0);
     a.base1 = static_cast<char*>(base1);
     a.stride_b = stride_b; a.stride_g = stride_g;
@@ -270,7 +262,7 @@ lvlm_status launch_inplace_compact(void* base0, void* base1, int64_t stride_b, i
     R = R / a.RL * a.RL;
     if (R < a.RL) R = a.RL;
     a.Rmax = R;
-    size_t smem = 2 * (size_t)R * Vsub * 16 + 3 * (size_t)R * 4;
+    size_t smem = 2 * (size_t)R * Vsub * 16 + 6 * (size_t)R * 4;
     const size_t red = ((size_t)a.RL + 1) * Vsub * 32;
     if (red > smem) smem = red;
     if (smem > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;

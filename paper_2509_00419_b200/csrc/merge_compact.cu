@@ -480,13 +480,13 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     } else {
         lvlm_status st = launch_inplace_compact(hidden, nullptr, hid_sb * 2, 0, d->B, 1, L.V,
                                                 L.Nout, src_map, wgt, meta, d->N, d->n, d->i0,
-                                                d->i0 + d->k, kMetaInts, stream);
+                                                d->i0 + d->k, kMetaInts, stream, 1, -1, nullptr, dst_map);
         if (st != LVLM_OK) return st;
     }
     if (Kc) {
         lvlm_status st = launch_inplace_compact(Kc, Vc, kv_sb * 2, kv_sh * 2, d->B, d->Hkv,
                                                 kHeadDim / 8, L.Nout, src_map, wgt, meta, d->N, d->n,
-                                                d->i0, d->i0 + d->k, kMetaInts, stream);
+                                                d->i0, d->i0 + d->k, kMetaInts, stream, 1, -1, nullptr, dst_map);
         if (st != LVLM_OK) return st;
     }
     return LVLM_OK;
