@@ -57,7 +57,7 @@ enum { LVLM_DEV_NONFINITE = 1, LVLM_DEV_TIMEOUT = 2, LVLM_DEV_BOUNDS = 4 };
  *                 the highest cosine similarity of the hidden rows (lower index wins ties),
  *                 weighted by the token masses; that layer's K and V rows are averaged with
  *                 the same assignment; no extra token.  Needs hidden_out (out of place),
- *                 1 <= k, n - k <= 131072, and a workspace sized with d->merge_mode set to it.
+ *                 1 <= k, n - k <= 65536, and a workspace sized with d->merge_mode set to it.
  *                 After the call the first B*(n-k) int32 of `ws` hold the assignment: for the
  *                 dropped tokens in ascending order, the index of their kept token in the
  *                 ascending list of kept tokens. */
@@ -144,7 +144,7 @@ lvlm_status lvlm_score_tokens(const void* Q, const void* K, const float* lse,
  *   near_tie  optional [B] int32 out: neighbours (p, p+1) of the order with p+1 >= k whose
  *             fp32 gap satisfies (s_p - s_{p+1}) < 1e-4 * |s_p|  (ties the caller may report)
  * -0 equals +0; NaN sorts last and sets LVLM_DEV_NONFINITE (so does an infinity).
- * Errors: INVALID_ARG (NULL score/rank, B<=0, n<=0, k outside [0,n]), UNSUPPORTED (n > 131072).
+ * Errors: INVALID_ARG (NULL score/rank, B<=0, n<=0, k outside [0,n]), UNSUPPORTED (n > 65536).
  */
 lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_stride, int k,
                              int32_t* rank, int32_t* kept_idx, int32_t* near_tie,

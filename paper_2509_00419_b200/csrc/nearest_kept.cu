@@ -607,7 +607,7 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(nk_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  kMaxDynSmem));
         st = launch_kernel_cluster(nk_group_kernel, dim3((L.r + kRankThreads - 1) / kRankThreads, S, d->B),
-                                   dim3(kRankThreads), (size_t)slice_len * 8, stream, dim3(1, S, 1),
+                                   dim3(kRankThreads), rank_smem_bytes(slice_len), stream, dim3(1, S, 1),
                                    best, L.r, d->k, S, slice_len, assign, order, sorted_t);
         if (st != LVLM_OK) return st;
         st = launch_kernel(nk_seg_kernel, dim3((d->k + 1 + 255) / 256, d->B), dim3(256), 0, stream, 1,

@@ -2,7 +2,10 @@
 // number of keys smaller than it.  Shared by token selection and by the grouping step of the
 // nearest-kept merge.  A CTA holds one slice of the keys in shared memory and every thread counts
 // for its own key; the CTAs of a cluster (one per slice, along y) add their counts through
-// distributed shared memory.
+// distributed shared memory.  A short slice is simply read through.  A long slice is first put into
+// 1024 bins by the high word of the key (linear between the slice's smallest and largest high word):
+// all keys of lower bins are smaller, so only the thread's own bin is read through.  How the keys
+// happen to be ordered inside a bin does not matter, the count is the same.
 #pragma once
 #include "common.cuh"
 
@@ -10,8 +13,15 @@ namespace lvlm {
 
 constexpr int kRankThreads = 256;
 constexpr int kRankMaxCluster = 8;
-constexpr int kRankMaxSlice = 16384;       // keys of one slice in shared memory (128 KB)
-constexpr int kRankMaxKeys = kRankMaxCluster * kRankMaxSlice;     // 131072 keys per sequence
+constexpr int kRankMaxSlice = 8192;        // keys of one slice in shared memory (twice 64 KB when binned)
+constexpr int kRankMaxKeys = kRankMaxCluster * kRankMaxSlice;     // 65536 keys per sequence
+constexpr int kRankBinFrom = 1024;         // slices at least this long are binned
+constexpr int kRankBins = 1024;
+
+// Shared memory a CTA needs for a slice of slice_len keys.
+inline size_t rank_smem_bytes(int slice_len) {
+    return slice_len >= kRankBinFrom ? (size_t)slice_len * 16 + (size_t)(2 * kRankBins + 2) * 4 : (size_t)slice_len * 8;
+}
 
 __device__ __forceinline__ uint32_t rank_cluster_rank() {
     uint32_t r;
@@ -57,11 +67,65 @@ __device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int
     const uint64_t kj = j < n ? key_of(j) : 0ull;
     __syncthreads();
     int cnt = 0;
-    const ulonglong2* sk2 = reinterpret_cast<const ulonglong2*>(sk);
+    if (slice_len >= kRankBinFrom) {
+        __shared__ uint32_t s_min[kRankThreads / 32], s_max[kRankThreads / 32];
+        __shared__ int s_scan[33];
+        uint64_t* sb = sk + slice_len;                                   // the keys again, bin by bin
+        int* start = reinterpret_cast<int*>(sb + slice_len);             // [kRankBins + 1]
+        int* cursor = start + kRankBins + 1;                             // [kRankBins]
+        const int nvalid = max(0, min(slice_len, n - i_lo));
+        // smallest and largest high word of the slice
+        uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+        for (int i = tid; i < nvalid; i += kRankThreads) {
+            const uint32_t h = (uint32_t)(sk[i] >> 32);
+            lo = min(lo, h); hi = max(hi, h);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            lo = min(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+            hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+        }
+        if ((tid & 31) == 0) { s_min[tid >> 5] = lo; s_max[tid >> 5] = hi; }
+        for (int i = tid; i <= kRankBins; i += kRankThreads) start[i] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int wv = 0; wv < kRankThreads / 32; ++wv) { lo = min(lo, s_min[wv]); hi = max(hi, s_max[wv]); }
+        const uint64_t span = (uint64_t)(hi - lo) + 1;                   // hi >= lo whenever the slice has keys
+        auto bin_of = [&](uint32_t h) { return (int)(((uint64_t)(h - lo) * kRankBins) / span); };
+        for (int i = tid; i < nvalid; i += kRankThreads) atomicAdd(&start[bin_of((uint32_t)(sk[i] >> 32))], 1);
+        __syncthreads();
+        {   // exclusive scan of the bin counts: four bins per thread
+            int c4[4], sum = 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { c4[u] = start[tid * 4 + u]; sum += c4[u]; }
+            int total;
+            int run = block_exclusive_scan(sum, s_scan, &total);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { start[tid * 4 + u] = run; cursor[tid * 4 + u] = run; run += c4[u]; }
+            if (tid == 0) start[kRankBins] = total;
+        }
+        __syncthreads();
+        for (int i = tid; i < nvalid; i += kRankThreads) {
+            const uint64_t key = sk[i];
+            sb[atomicAdd(&cursor[bin_of((uint32_t)(key >> 32))], 1)] = key;
+        }
+        __syncthreads();
+        const uint32_t hj = (uint32_t)(kj >> 32);
+        if (nvalid > 0 && j < n) {
+            if (hj > hi) cnt = nvalid;
+            else if (hj >= lo) {
+                const int bj = bin_of(hj);
+                cnt = start[bj];
+                for (int p = start[bj]; p < start[bj + 1]; ++p) cnt += sb[p] < kj;
+            }
+        }
+    } else {
+        const ulonglong2* sk2 = reinterpret_cast<const ulonglong2*>(sk);
 #pragma unroll 4
-    for (int i = 0; i < slice_len / 2; ++i) {
-        const ulonglong2 v = sk2[i];
-        cnt += (v.x < kj) + (v.y < kj);
+        for (int i = 0; i < slice_len / 2; ++i) {
+            const ulonglong2 v = sk2[i];
+            cnt += (v.x < kj) + (v.y < kj);
+        }
     }
     if (S == 1) { *count = cnt; return j < n; }
     s_cnt[tid] = cnt;

@@ -96,7 +96,7 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     {
         const lvlm_status st = launch_kernel_cluster(select_count_kernel, dim3((n + kRankThreads - 1) / kRankThreads, S, B),
-                                                     dim3(kRankThreads), (size_t)slice_len * 8, stream, dim3(1, S, 1),
+                                                     dim3(kRankThreads), rank_smem_bytes(slice_len), stream, dim3(1, S, 1),
                                                      score, score_stride, n, S, slice_len, rank, dev_status);
         if (st != LVLM_OK) return st;
     }

@@ -77,7 +77,7 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     sel = lambda n, k, s=p, r=p: lib.lvlm_select_topk(s, 1, n, 0, k, r, None, None, None, 0, None, None)
     assert sel(10, 11) == L.ERR_INVALID_ARG and sel(10, -1) == L.ERR_INVALID_ARG
     assert sel(0, 0) == L.ERR_INVALID_ARG and sel(10, 5, s=None) == L.ERR_INVALID_ARG
-    assert sel(131073, 5) == L.ERR_UNSUPPORTED
+    assert sel(65537, 5) == L.ERR_UNSUPPORTED
 
     def merge(dd, h=p, rk=p, Kc=None, Vc=None, mode=0, wc=None, w=ws, wn=n_ws):
         return lib.lvlm_merge_compact(h, None, Kc, Vc, None, rk, ref(dd), mode, wc, None, None, w, wn, None, None)
