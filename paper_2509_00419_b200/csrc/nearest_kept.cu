@@ -157,10 +157,10 @@ nk_norm_kernel(const uint4* __restrict__ out, int64_t out_stride_b, int V, int i
 // dropped tokens, S, B), clusters (1, S, 1).  Writes the assignment, the sorted order and the kept
 // token at every place of that order; a second kernel finds where every kept token's segment starts.
 __global__ void __launch_bounds__(kRankThreads)
-nk_group_kernel(const unsigned long long* __restrict__ best, int r, int k, int S, int slice_len,
+nk_group_kernel(const unsigned long long* __restrict__ best, int r, int k, int S, int slice_len, int jt,
                 int32_t* __restrict__ assign, int32_t* __restrict__ order, int32_t* __restrict__ sorted_t) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ int s_cnt[kRankThreads];
+    __shared__ int s_cnt[kRankMaxJT * kRankThreads];
     pdl_enter();
     const int b = blockIdx.z;
     const unsigned long long* bb = best + (int64_t)b * r;
@@ -168,13 +168,18 @@ nk_group_kernel(const unsigned long long* __restrict__ best, int r, int k, int S
         const uint32_t t = 0xFFFFFFFFu - (uint32_t)(bb[q] & 0xFFFFFFFFull);
         return ((uint64_t)(t < (uint32_t)k ? t : 0u) << 32) | (uint32_t)q;     // nothing won: kept token 0
     };
-    int p = 0;
-    if (rank_by_counting(key_of, r, S, slice_len, reinterpret_cast<uint64_t*>(smem_raw), s_cnt, &p)) {
-        const int q = blockIdx.x * kRankThreads + threadIdx.x;
-        const int t = (int)(key_of(q) >> 32);
-        assign[(int64_t)b * r + q] = t;
-        order[(int64_t)b * r + p] = q;
-        sorted_t[(int64_t)b * r + p] = t;
+    int p[kRankMaxJT];
+    if (rank_by_counting(key_of, r, S, slice_len, jt, reinterpret_cast<uint64_t*>(smem_raw), s_cnt, p)) {
+#pragma unroll
+        for (int u = 0; u < kRankMaxJT; ++u) {
+            const int q = rank_key_index(jt, u);
+            if (u < jt && q < r) {
+                const int t = (int)(key_of(q) >> 32);
+                assign[(int64_t)b * r + q] = t;
+                order[(int64_t)b * r + p[u]] = q;
+                sorted_t[(int64_t)b * r + p[u]] = t;
+            }
+        }
     }
 }
 
@@ -602,13 +607,13 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
         if (st != LVLM_OK) return st;
     }
     {
-        int S, slice_len;
-        rank_shape(L.r, d->B, &S, &slice_len);
+        int S, slice_len, jt;
+        rank_shape(L.r, d->B, &S, &slice_len, &jt);
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(nk_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  kMaxDynSmem));
-        st = launch_kernel_cluster(nk_group_kernel, dim3((L.r + kRankThreads - 1) / kRankThreads, S, d->B),
+        st = launch_kernel_cluster(nk_group_kernel, dim3((L.r + kRankThreads * jt - 1) / (kRankThreads * jt), S, d->B),
                                    dim3(kRankThreads), rank_smem_bytes(slice_len), stream, dim3(1, S, 1),
-                                   best, L.r, d->k, S, slice_len, assign, order, sorted_t);
+                                   best, L.r, d->k, S, slice_len, jt, assign, order, sorted_t);
         if (st != LVLM_OK) return st;
         st = launch_kernel(nk_seg_kernel, dim3((d->k + 1 + 255) / 256, d->B), dim3(256), 0, stream, 1,
                            sorted_t, L.r, d->k, seg);

@@ -17,6 +17,7 @@ constexpr int kRankMaxSlice = 8192;        // keys of one slice in shared memory
 constexpr int kRankMaxKeys = kRankMaxCluster * kRankMaxSlice;     // 65536 keys per sequence
 constexpr int kRankBinFrom = 1024;         // slices at least this long are binned
 constexpr int kRankBins = 1024;
+constexpr int kRankMaxJT = 4;              // keys a thread ranks when the slices are binned (bins are built once per CTA)
 
 // Shared memory a CTA needs for a slice of slice_len keys.
 inline size_t rank_smem_bytes(int slice_len) {
@@ -42,20 +43,25 @@ __device__ __forceinline__ int rank_ld_cluster(const int* my_smem, uint32_t rank
 
 // Number of slices (cluster size) and keys per slice for n keys in each of B sequences: up to eight
 // CTAs of 256 threads per SM, at least 256 keys per slice; the slice length is even.
-inline void rank_shape(int n, int B, int* S, int* slice_len) {
+inline void rank_shape(int n, int B, int* S, int* slice_len, int* jt) {
     const int jblocks = (n + kRankThreads - 1) / kRankThreads;
     int s = 1;
     while (s < kRankMaxCluster && (int64_t)jblocks * B * (2 * s) <= 8 * 148 && n / (2 * s) >= 256) s *= 2;
     while (s < kRankMaxCluster && (n + s - 1) / s > kRankMaxSlice) s *= 2;       // a slice has to fit
     *S = s;
     *slice_len = (((n + s - 1) / s) + 1) & ~1;
+    *jt = *slice_len >= 4096 ? kRankMaxJT : 1;           // few CTAs per slice when a slice is costly to bin
 }
 
-// Call from every thread of a CTA of kRankThreads threads in a grid (key blocks, S, B) with clusters
-// (1, S, 1).  key_of(i) gives key i of this sequence (i < n).  Returns true in the threads that hold a
-// final count (*count = number of keys smaller than key j, j = blockIdx.x * 256 + threadIdx.x < n).
+// Call from every thread of a CTA of kRankThreads threads in a grid (ceil(n / (256 jt)), S, B) with
+// clusters (1, S, 1).  key_of(i) gives key i of this sequence (i < n).  A thread ranks the jt keys
+// j_u = rank_key_index(u) = (blockIdx.x * jt + u) * 256 + threadIdx.x.  Returns true in the threads that
+// hold final counts (count[u] = number of keys smaller than key j_u, for the j_u < n).
+// s_cnt: kRankMaxJT * kRankThreads ints of shared memory.
+__device__ __forceinline__ int rank_key_index(int jt, int u) { return (blockIdx.x * jt + u) * kRankThreads + threadIdx.x; }
+
 template <typename KeyFn>
-__device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int slice_len, uint64_t* sk,
+__device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int slice_len, int jt, uint64_t* sk,
                                                  int* s_cnt, int* count) {
     const int s = (int)rank_cluster_rank(), tid = threadIdx.x;
     const int i_lo = s * slice_len;
@@ -63,10 +69,14 @@ __device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int
         const int gi = i_lo + i;
         sk[i] = gi < n ? key_of(gi) : ~0ull;              // padding sorts after every real key
     }
-    const int j = blockIdx.x * kRankThreads + tid;
-    const uint64_t kj = j < n ? key_of(j) : 0ull;
+    uint64_t kjs[kRankMaxJT];
+#pragma unroll
+    for (int u = 0; u < kRankMaxJT; ++u) {
+        const int j = rank_key_index(jt, u);
+        kjs[u] = (u < jt && j < n) ? key_of(j) : 0ull;
+        count[u] = 0;
+    }
     __syncthreads();
-    int cnt = 0;
     if (slice_len >= kRankBinFrom) {
         __shared__ uint32_t s_min[kRankThreads / 32], s_max[kRankThreads / 32];
         __shared__ int s_scan[33];
@@ -110,32 +120,45 @@ __device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int
             sb[atomicAdd(&cursor[bin_of((uint32_t)(key >> 32))], 1)] = key;
         }
         __syncthreads();
-        const uint32_t hj = (uint32_t)(kj >> 32);
-        if (nvalid > 0 && j < n) {
-            if (hj > hi) cnt = nvalid;
-            else if (hj >= lo) {
-                const int bj = bin_of(hj);
-                cnt = start[bj];
-                for (int p = start[bj]; p < start[bj + 1]; ++p) cnt += sb[p] < kj;
+#pragma unroll
+        for (int u = 0; u < kRankMaxJT; ++u) {
+            const uint64_t kj = kjs[u];
+            const uint32_t hj = (uint32_t)(kj >> 32);
+            int cnt = 0;
+            if (nvalid > 0 && u < jt && rank_key_index(jt, u) < n) {
+                if (hj > hi) cnt = nvalid;
+                else if (hj >= lo) {
+                    const int bj = bin_of(hj);
+                    cnt = start[bj];
+                    for (int p = start[bj]; p < start[bj + 1]; ++p) cnt += sb[p] < kj;
+                }
             }
+            count[u] = cnt;
         }
     } else {
+        const uint64_t kj = kjs[0];                       // short slices: one key per thread (jt == 1)
+        int cnt = 0;
         const ulonglong2* sk2 = reinterpret_cast<const ulonglong2*>(sk);
 #pragma unroll 4
         for (int i = 0; i < slice_len / 2; ++i) {
             const ulonglong2 v = sk2[i];
             cnt += (v.x < kj) + (v.y < kj);
         }
+        count[0] = cnt;
     }
-    if (S == 1) { *count = cnt; return j < n; }
-    s_cnt[tid] = cnt;
+    if (S == 1) return true;
+#pragma unroll
+    for (int u = 0; u < kRankMaxJT; ++u) s_cnt[u * kRankThreads + tid] = count[u];
     rank_cluster_barrier();
-    bool mine = false;
-    if (s == 0 && j < n) {
-        int tot = 0;
-        for (int r = 0; r < S; ++r) tot += rank_ld_cluster(&s_cnt[tid], r);
-        *count = tot;
-        mine = true;
+    const bool mine = s == 0;
+    if (mine) {
+#pragma unroll
+        for (int u = 0; u < kRankMaxJT; ++u) {
+            int tot = 0;
+            if (u < jt)
+                for (int r = 0; r < S; ++r) tot += rank_ld_cluster(&s_cnt[u * kRankThreads + tid], r);
+            count[u] = tot;
+        }
     }
     rank_cluster_barrier();                               // nobody leaves while its counts are read
     return mine;

@@ -14,20 +14,25 @@
 
 namespace lvlm {
 
-// grid (blocks of 256 tokens, S, B), clusters (1, S, 1).
+// grid (blocks of 256 jt tokens, S, B), clusters (1, S, 1).
 __global__ void __launch_bounds__(kRankThreads)
-select_count_kernel(const float* __restrict__ score, int64_t stride, int n, int S, int slice_len,
+select_count_kernel(const float* __restrict__ score, int64_t stride, int n, int S, int slice_len, int jt,
                     int32_t* __restrict__ rank, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ int s_cnt[kRankThreads];
+    __shared__ int s_cnt[kRankMaxJT * kRankThreads];
     pdl_enter();
     const int b = blockIdx.z;
     const float* row = score + (int64_t)b * stride;
     bool nonfinite = false;
     auto key_of = [&](int i) { return ((uint64_t)desc_key(row[i], &nonfinite) << 32) | (uint32_t)i; };
-    int cnt = 0;
-    const bool mine = rank_by_counting(key_of, n, S, slice_len, reinterpret_cast<uint64_t*>(smem_raw), s_cnt, &cnt);
-    if (mine) rank[(int64_t)b * n + blockIdx.x * kRankThreads + threadIdx.x] = cnt;
+    int cnt[kRankMaxJT];
+    if (rank_by_counting(key_of, n, S, slice_len, jt, reinterpret_cast<uint64_t*>(smem_raw), s_cnt, cnt)) {
+#pragma unroll
+        for (int u = 0; u < kRankMaxJT; ++u) {
+            const int j = rank_key_index(jt, u);
+            if (u < jt && j < n) rank[(int64_t)b * n + j] = cnt[u];
+        }
+    }
     // every key is looked at by the CTAs of slice 0 as "their own" key: one report is enough
     if (nonfinite && blockIdx.y == 0 && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
 }
@@ -90,14 +95,14 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
     if (score_stride == 0) score_stride = n;
     if (score_stride < n) return LVLM_ERR_INVALID_ARG;
     if (n > kRankMaxKeys) return LVLM_ERR_UNSUPPORTED;
-    int S, slice_len;
-    rank_shape(n, B, &S, &slice_len);
+    int S, slice_len, jt;
+    rank_shape(n, B, &S, &slice_len, &jt);
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_count_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     {
-        const lvlm_status st = launch_kernel_cluster(select_count_kernel, dim3((n + kRankThreads - 1) / kRankThreads, S, B),
+        const lvlm_status st = launch_kernel_cluster(select_count_kernel, dim3((n + kRankThreads * jt - 1) / (kRankThreads * jt), S, B),
                                                      dim3(kRankThreads), rank_smem_bytes(slice_len), stream, dim3(1, S, 1),
-                                                     score, score_stride, n, S, slice_len, rank, dev_status);
+                                                     score, score_stride, n, S, slice_len, jt, rank, dev_status);
         if (st != LVLM_OK) return st;
     }
     if (!kept_idx && !near_tie) return LVLM_OK;
