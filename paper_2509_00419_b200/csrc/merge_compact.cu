@@ -94,7 +94,29 @@ __device__ __forceinline__ float merge_weight(int mode, int p, int r1, float inv
     }
 }
 
-// One CTA per sequence: source map, weights, position ids, new length.
+__device__ __forceinline__ uint32_t plan_cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void plan_cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ int plan_ld_cluster(const int* my_smem, uint32_t rank) {
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    int v;
+    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+// A cluster of P CTAs per sequence (grid (P, B)): source map, destination map, weights, position ids,
+// new length.  CTA r takes the r-th run of the image tokens: it counts its kept tokens, learns from the
+// lower ranks how many came before, then writes the maps of its run (tile by tile, thread = token,
+// coalesced).  The position ids are compacted in place in rounds of P x blockDim output rows: every CTA
+// loads its rows of the round, a cluster barrier, then it stores them (a row's source lies at or behind it,
+// so nothing a later round needs is overwritten).
 __global__ void __launch_bounds__(1024)
 merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int i0, int n, int k,
                   int mode, float inv_sum, const float* __restrict__ w_custom,
@@ -103,15 +125,17 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
                   int32_t* dev_status) {
     __shared__ int scan_scratch[33];
     __shared__ float fsum_scratch[33];
-    __shared__ int s_first_drop, s_merged_tok, s_pos_new;
+    __shared__ int s_total, s_first_drop, s_merged_tok;
     pdl_enter();
-    const int b = blockIdx.x;
+    const int b = blockIdx.y, P = (int)gridDim.x, cr = (int)plan_cluster_rank();
     const int r1 = n - k, r = r1 - 1, Nout = N - r;
     const int32_t* rk = rank + (int64_t)b * n;
     int32_t* src = src_map + (int64_t)b * N;
     int32_t* dst = dst_map + (int64_t)b * N;      // output row of every input row, -1 = merged away
     float* w = wgt + (int64_t)b * n;
-    if (threadIdx.x == 0) { s_first_drop = n; s_merged_tok = 0; }
+    const int chunk = (n + P - 1) / P;
+    const int c_lo = min(n, cr * chunk), c_hi = min(n, c_lo + chunk);
+    if (threadIdx.x == 0) { s_total = 0; s_first_drop = n; s_merged_tok = -1; }
 
     if (mode == LVLM_W_CUSTOM) {
         float part = 0.f;
@@ -121,17 +145,34 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
     }
     __syncthreads();
 
-    // tile by tile, thread = token of the tile (coalesced), running count of the kept tokens so far
+    // kept tokens of my run
     bool bad = false;
-    int kept_before = 0;
-    for (int t0 = 0; t0 < n; t0 += blockDim.x) {
+    int mine = 0;
+    for (int t0 = c_lo; t0 < c_hi; t0 += blockDim.x) {
         const int j = t0 + threadIdx.x;
-        const int rj = j < n ? rk[j] : n;                 // past the end: counts as dropped, writes nothing
-        if (j < n && (rj < 0 || rj >= n)) bad = true;
-        const int is_kept = j < n && rj < k;
+        const int rj = j < c_hi ? rk[j] : n;
+        if (j < c_hi && (rj < 0 || rj >= n)) bad = true;
+        mine += j < c_hi && rj < k;
+    }
+    mine = warp_sum(mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_total, mine);
+    plan_cluster_barrier();
+    int kept_before = 0, kept_all = 0;
+    for (int q = 0; q < P; ++q) {
+        const int t = plan_ld_cluster(&s_total, q);
+        kept_before += q < cr ? t : 0;
+        kept_all += t;
+    }
+    if (kept_all != k) bad = true;
+
+    // the maps of my run
+    for (int t0 = c_lo; t0 < c_hi; t0 += blockDim.x) {
+        const int j = t0 + threadIdx.x;
+        const int rj = j < c_hi ? rk[j] : n;              // past the end: counts as dropped, writes nothing
+        const int is_kept = j < c_hi && rj < k;
         int total;
         const int off = kept_before + block_exclusive_scan(is_kept, scan_scratch, &total);
-        if (j < n) {
+        if (j < c_hi) {
             float wj = 0.f;
             if (is_kept) {
                 if (off < k) src[i0 + off] = i0 + j;
@@ -145,39 +186,44 @@ merge_plan_kernel(const int32_t* __restrict__ rank, int32_t* pos_ids, int N, int
             }
             w[j] = wj;
         }
-        int fd = (j < n && !is_kept) ? j : n;              // first dropped token: one atomic per warp
+        int fd = (j < c_hi && !is_kept) ? j : n;           // first dropped token: one atomic per warp
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) fd = min(fd, __shfl_xor_sync(0xFFFFFFFFu, fd, o));
         if ((threadIdx.x & 31) == 0 && fd < n) atomicMin(&s_first_drop, fd);
         kept_before += total;
     }
-    if (kept_before != k) bad = true;
-    for (int o = threadIdx.x; o < Nout; o += blockDim.x) {
+    // rows outside the image span, shared out over the CTAs
+    for (int o = cr * blockDim.x + threadIdx.x; o < Nout; o += P * blockDim.x) {
         if (o < i0) { src[o] = o; dst[o] = o; }
         else if (o == i0 + k) src[o] = -1;
         else if (o > i0 + k) { src[o] = o + r; dst[o + r] = o; }
     }
     if (bad && dev_status) atomicOr(dev_status, LVLM_DEV_BOUNDS);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        meta[b * kMetaInts + 0] = i0 + s_first_drop;     // first row whose content changes
+    plan_cluster_barrier();                               // the maps are complete, every CTA's findings are in place
+    int first_drop = n, merged_tok = 0;
+    for (int q = 0; q < P; ++q) {
+        first_drop = min(first_drop, plan_ld_cluster(&s_first_drop, q));
+        const int mt = plan_ld_cluster(&s_merged_tok, q);
+        if (mt >= 0) merged_tok = mt;
+    }
+    if (cr == 0 && threadIdx.x == 0) {
+        meta[b * kMetaInts + 0] = i0 + first_drop;       // first row whose content changes
         meta[b * kMetaInts + 1] = 0;                     // ticket counter of the merge blocks
-        meta[b * kMetaInts + 2] = s_merged_tok;
+        meta[b * kMetaInts + 2] = merged_tok;
         if (new_len) new_len[b] = Nout;
-        if (pos_ids) s_pos_new = pos_ids[(int64_t)b * N + i0 + s_merged_tok];
     }
     if (pos_ids) {
-        // in place, tile by tile in increasing order: a tile's sources lie at or after it
         int32_t* pid = pos_ids + (int64_t)b * N;
-        for (int o0 = 0; o0 < Nout; o0 += blockDim.x) {
-            const int o = o0 + threadIdx.x;
+        const int pos_new = pid[i0 + merged_tok];         // read before any CTA stores (first store: after a barrier)
+        for (int o0 = 0; o0 < Nout; o0 += P * blockDim.x) {
+            const int o = o0 + cr * blockDim.x + threadIdx.x;
             int val = 0;
-            __syncthreads();
-            if (o < Nout) { const int s = src[o]; val = s >= 0 ? pid[s] : s_pos_new; }
-            __syncthreads();
+            if (o < Nout) { const int sidx = src[o]; val = sidx >= 0 ? pid[sidx] : pos_new; }
+            plan_cluster_barrier();
             if (o < Nout) pid[o] = val;
         }
     }
+    plan_cluster_barrier();                               // nobody leaves while its shared memory may still be read
 }
 
 __global__ void identity_len_kernel(int32_t* new_len, int B, int N) {
@@ -467,7 +513,9 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     else if (mode == LVLM_W_UNIFORM) inv_sum = (float)(1.0 / (double)L.r1);
     const int plan_threads = d->n >= 1024 ? 1024 : (d->n <= 128 ? 128 : ((d->n + 31) / 32) * 32);
     {
-        const lvlm_status st = launch_kernel(merge_plan_kernel, dim3(d->B), dim3(plan_threads), 0, stream, 1,
+        int P = (d->n + 2047) / 2048;                    // CTAs per sequence: at least two tiles of tokens each
+        P = P < 1 ? 1 : (P > 8 ? 8 : P);
+        const lvlm_status st = launch_kernel(merge_plan_kernel, dim3(P, d->B), dim3(plan_threads), 0, stream, P,
                                              rank, pos_ids, d->N, d->i0, d->n, d->k, (int)mode, inv_sum, w_custom,
                                              src_map, dst_map, wgt, meta, new_len, dev_status);
         if (st != LVLM_OK) return st;
