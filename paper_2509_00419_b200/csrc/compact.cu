@@ -44,6 +44,12 @@ __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n"
                  "barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
+// Execution barrier only: nobody passes before everybody has arrived, but no memory is published.  Enough
+// between "my rows are on chip" and "I overwrite rows": nobody reads what another CTA writes here.
+__device__ __forceinline__ void cluster_barrier_exec() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;\n"
+                 "barrier.cluster.wait.aligned;\n" ::: "memory");
+}
 __device__ __forceinline__ float ld_cluster_f32(const float* my_smem, uint32_t rank) {
     uint32_t local = (uint32_t)__cvta_generic_to_shared(my_smem), remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
@@ -160,7 +166,8 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
         float regw[kIdxPerThread];
         fetch_idx(t0 + 2 * Rc, reg, regw);            // in flight while this round runs
         cp_async_wait_group<1>();                     // this super-tile's rows have landed
-        cluster_barrier();                            // ... in every CTA of the cluster
+        __syncthreads();                              // ... for every thread of this CTA
+        cluster_barrier_exec();                       // ... in every CTA of the cluster
         const uint4* cur = buf[k & 1];
         const int32_t* cur_idx = s_idx + (k % 3) * a.Rmax;
         const float* cur_wt = s_wt + (k % 3) * a.Rmax;
