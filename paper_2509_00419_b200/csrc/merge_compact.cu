@@ -20,7 +20,7 @@ struct MergeLayout {
 
 constexpr int kHidThreads = 256;       // streaming kernel: thread = 16-byte column group (+256, +512 ...)
 constexpr int kHidMaxChunks = 4;       // column groups per thread: rows up to 4 * 256 * 8 = 8192 channels
-constexpr int kNoRow = -2147483647 - 1;  // marks a slot of the four-row group that lies past the CTA's rows
+constexpr int kNoRow = -2147483647 - 1;  // marks a slot of a row group that lies past the last row
 constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
 
 // One wave of CTAs over the whole batch (four per SM fit for rows up to 4096 channels, two beyond:
@@ -258,7 +258,7 @@ __device__ __forceinline__ float4 hid_ld_cluster_f4(const float* my_smem, uint32
 }
 
 // Hidden states, out of place.  grid (CTAs per sequence, B), clusters of `cl` CTAs along x.  A CTA
-// takes every grid.x-th group of four consecutive INPUT rows and reads each row exactly once: a kept
+// takes every grid.x-th group of two consecutive INPUT rows and reads each row exactly once: a kept
 // row goes to its destination, a merged row is added, times its weight, to fp32 sums the thread
 // keeps for its columns (its rows in increasing order).  The CTAs of a cluster add their sums in rank
 // order through distributed shared memory and park one partial per cluster; the last cluster of
@@ -288,14 +288,13 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
 
-    // groups of four rows are dealt out round robin, so that every CTA gets the same mix of kept
-    // rows (read and written) and merged rows (read only)
-    for (int ib = cta * 4; ib < i_hi; ib += (int)gridDim.x * 4) {
-        int d[4];
-        float wj[4];
-        uint4 x[4][CH];
+    // Groups of kG rows are dealt out round robin, so that every CTA gets the same mix of kept rows (read
+    // and written) and merged rows (read only).  Two groups are in flight in turn: the loads of the next
+    // one are issued before the current one is used.
+    constexpr int kG = 2;
+    auto load_group = [&](int ib, int* d, float* wj, uint4 (*x)[CH]) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kG; ++u) {
             const int i = ib + u;
             d[u] = i < i_hi ? dst[i] : kNoRow;
             wj[u] = (w && i < i_hi && i >= i0 && i < i0 + n) ? w[i] : 0.f;
@@ -305,8 +304,10 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
                 x[u][ci] = (i < i_hi && c < V) ? __ldg(hin + (int64_t)i * V + c) : make_uint4(0, 0, 0, 0);
             }
         }
+    };
+    auto use_group = [&](const int* d, const float* wj, const uint4 (*x)[CH]) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kG; ++u) {
             if (d[u] >= 0) {
 #pragma unroll
                 for (int ci = 0; ci < CH; ++ci) {
@@ -330,6 +331,20 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
                     acc[ci][6] = fmaf(wj[u], bf16_lo(x[u][ci].w), acc[ci][6]); acc[ci][7] = fmaf(wj[u], bf16_hi(x[u][ci].w), acc[ci][7]);
                 }
             }
+        }
+    };
+    {
+        const int step = (int)gridDim.x * kG;
+        int dA[kG], dB[kG];
+        float wA[kG], wB[kG];
+        uint4 xA[kG][CH], xB[kG][CH];
+        int ib = cta * kG;
+        load_group(ib, dA, wA, xA);
+        for (; ib < i_hi; ib += 2 * step) {
+            load_group(ib + step, dB, wB, xB);
+            use_group(dA, wA, xA);
+            load_group(ib + 2 * step, dA, wA, xA);
+            use_group(dB, wB, xB);
         }
     }
 
