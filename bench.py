@@ -32,7 +32,7 @@ import torch
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from one ncu capture of the kernel as it stands
 # (set back to None whenever that kernel changes); the capture and its command are in the named file
 NCU_TRAFFIC = {
-    ("cfg2", "lvlm_decode_attn"): {"bytes_per_launch": 1750263, "source": "profiles/decode_cluster_kernel_step_cfg2.txt"},
+    ("cfg2", "lvlm_decode_attn"): {"bytes_per_launch": 1749979, "source": "profiles/decode_cluster_kernel_step_cfg2.txt"},
 }
 DOMINANT_KERNEL = {"lvlm_decode_attn": "decode_cluster_kernel", "lvlm_score_tokens": "score_tc_kernel<0> + <1>",
                    "lvlm_merge_compact": "merge_plan + hidden_stream + inplace_compact kernels",

@@ -528,7 +528,7 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     else if (mode == LVLM_W_UNIFORM) inv_sum = (float)(1.0 / (double)L.r1);
     const int plan_threads = d->n >= 1024 ? 1024 : (d->n <= 128 ? 128 : ((d->n + 31) / 32) * 32);
     {
-        int P = (d->n + 2047) / 2048;                    // CTAs per sequence: at least two tiles of tokens each
+        int P = (d->n + 4095) / 4096;                    // CTAs per sequence: about four tiles of tokens each
         P = P < 1 ? 1 : (P > 8 ? 8 : P);
         const lvlm_status st = launch_kernel(merge_plan_kernel, dim3(P, d->B), dim3(plan_threads), 0, stream, P,
                                              rank, pos_ids, d->N, d->i0, d->n, d->k, (int)mode, inv_sum, w_custom,
