@@ -80,14 +80,80 @@ __device__ __forceinline__ unsigned long long ceil_muldiv(unsigned long long a, 
     return q + (rem != 0);
 }
 
+constexpr int kPlanBins = 1024;
+constexpr int kPlanBinFrom = 512;          // evictable sets at least this large are ordered by binned counting
+constexpr int kPlanBinMaxCap = 8192;       // ... when the second key array fits in shared memory
+
+// Ascending order of m distinct 64-bit keys (m <= blockDim.x * 16) without a sorting network: the keys
+// are put into 1024 bins by their high word (linear between the extremes), the place of a key is the
+// number of keys in lower bins plus the number of smaller keys in its own bin.  On return `sorted` holds
+// the keys in order.  srank: m ints, bins: 2 * kPlanBins + 1 ints of shared memory.
+__device__ __forceinline__ void block_order_by_bins(const uint64_t* keys, uint64_t* sorted, int m, int* srank,
+                                                    int* bins, int* scan_scratch) {
+    __shared__ uint32_t s_min[32], s_max[32];
+    int* start = bins;                       // [kPlanBins + 1]
+    int* cursor = bins + kPlanBins + 1;      // [kPlanBins]
+    const int tid = threadIdx.x;
+    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+    for (int i = tid; i < m; i += blockDim.x) {
+        const uint32_t h = (uint32_t)(keys[i] >> 32);
+        lo = min(lo, h); hi = max(hi, h);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = min(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+        hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    if ((tid & 31) == 0) { s_min[tid >> 5] = lo; s_max[tid >> 5] = hi; }
+    for (int i = tid; i <= kPlanBins; i += blockDim.x) start[i] = 0;
+    __syncthreads();
+    for (int wv = 0; wv < (int)(blockDim.x >> 5); ++wv) { lo = min(lo, s_min[wv]); hi = max(hi, s_max[wv]); }
+    const uint64_t span = (uint64_t)(hi - lo) + 1;
+    auto bin_of = [&](uint32_t h) { return (int)(((uint64_t)(h - lo) * kPlanBins) / span); };
+    for (int i = tid; i < m; i += blockDim.x) atomicAdd(&start[bin_of((uint32_t)(keys[i] >> 32))], 1);
+    __syncthreads();
+    {   // exclusive scan of the bin counts: the first 256 threads take four bins each
+        int c4[4] = {0, 0, 0, 0}, sum = 0;
+        if (tid < kPlanBins / 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { c4[u] = start[tid * 4 + u]; sum += c4[u]; }
+        }
+        int total;
+        int run = block_exclusive_scan(sum, scan_scratch, &total);
+        if (tid < kPlanBins / 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { start[tid * 4 + u] = run; cursor[tid * 4 + u] = run; run += c4[u]; }
+        }
+        if (tid == 0) start[kPlanBins] = total;
+    }
+    __syncthreads();
+    for (int i = tid; i < m; i += blockDim.x) {
+        const uint64_t key = keys[i];
+        sorted[atomicAdd(&cursor[bin_of((uint32_t)(key >> 32))], 1)] = key;       // bin by bin, any order inside
+    }
+    __syncthreads();
+    for (int i = tid; i < m; i += blockDim.x) {
+        const uint64_t key = keys[i];
+        const int bj = bin_of((uint32_t)(key >> 32));
+        int r = start[bj];
+        for (int p = start[bj]; p < start[bj + 1]; ++p) r += sorted[p] < key;
+        srank[i] = r;
+    }
+    __syncthreads();
+    for (int i = tid; i < m; i += blockDim.x) sorted[srank[i]] = keys[i];
+    __syncthreads();
+}
+
 __global__ void __launch_bounds__(1024)
 kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __restrict__ e_lo,
-               const int32_t* __restrict__ e_hi, int Hkv, int cap, int recent, int P_max,
+               const int32_t* __restrict__ e_hi, int Hkv, int cap, int recent, int P_max, int binned,
                unsigned long long beta_ppm, int budget, int32_t* __restrict__ src_map,
                int32_t* __restrict__ meta, int32_t* __restrict__ nout, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* keys = reinterpret_cast<uint64_t*>(smem_raw);
     int32_t* flag = reinterpret_cast<int32_t*>(keys + P_max);      // [cap]
+    uint64_t* keys2 = reinterpret_cast<uint64_t*>(flag + ((cap + 1) & ~1));            // [P_max], binned only
+    int32_t* bins = reinterpret_cast<int32_t*>(keys2 + P_max);                         // [2 * kPlanBins + 1]
     __shared__ int scan_scratch[33];
     __shared__ long long scan_ll[33];
     __shared__ unsigned long long s_thr;
@@ -124,7 +190,12 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
     }
     if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
     __syncthreads();
-    block_bitonic_sort(keys, P);
+    if (binned && m >= kPlanBinFrom) {
+        block_order_by_bins(keys, keys2, m, flag, bins, scan_scratch);
+        keys = keys2;
+    } else {
+        block_bitonic_sort(keys, P);
+    }
 
     // ---- how many entries of E reach the threshold ---------------------------------------
     int k_beta = m;
@@ -221,12 +292,14 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
     const int P_max = next_pow2(d->cap < 2 ? 2 : d->cap);
     int threads = P_max / 2;
     threads = threads < 64 ? 64 : (threads > 1024 ? 1024 : threads);
-    const size_t smem = (size_t)P_max * 8 + (size_t)d->cap * 4;
+    const int binned = d->cap >= kPlanBinFrom && d->cap <= kPlanBinMaxCap;
+    const size_t smem = (size_t)P_max * 8 + (size_t)((d->cap + 1) & ~1) * 4 +
+                        (binned ? (size_t)P_max * 8 + (size_t)(2 * kPlanBins + 2) * 4 : 0);
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(kv_plan_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     {
         const lvlm_status st = launch_kernel(kv_plan_kernel, dim3(d->Hkv, d->B), dim3(threads), smem, stream, 1,
-                                             acc_score, pos, len, e_lo, e_hi, d->Hkv, d->cap, d->recent, P_max,
+                                             acc_score, pos, len, e_lo, e_hi, d->Hkv, d->cap, d->recent, P_max, binned,
                                              beta_ppm, budget, src_map, meta, nout, dev_status);
         if (st != LVLM_OK) return st;
     }
