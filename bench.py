@@ -653,8 +653,9 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "layers": w.L, "hidden": w.C, "heads": f"{w.H}/{w.Hkv}",
-                   "image_tokens": w.n, "text_tokens": w.T,
+        "config": {"workload": w.name,
+                   "shape": "%d sequence(s) x (%d image + %d text tokens), %d channels, %d/%d query/KV heads of 128, %d layers"
+                            % (w.B, w.n, w.T, w.C, w.H, w.Hkv, w.L),
                    "stages": [[l, m] for l, m in w.stages], "beta": w.beta,
                    "l2": "flushed between timed iterations (384 MB overwrite)",
                    "step": "reduce stages + score/compress layers %d..%d + one decode step over %d layers"
