@@ -144,7 +144,8 @@ lvlm_status lvlm_score_tokens(const void* Q, const void* K, const float* lse,
  *   near_tie  optional [B] int32 out: neighbours (p, p+1) of the order with p+1 >= k whose
  *             fp32 gap satisfies (s_p - s_{p+1}) < 1e-4 * |s_p|  (ties the caller may report)
  * -0 equals +0; NaN sorts last and sets LVLM_DEV_NONFINITE (so does an infinity).
- * Errors: INVALID_ARG (NULL score/rank, B<=0, n<=0, k outside [0,n]), UNSUPPORTED (n > 65536).
+ * Errors: INVALID_ARG (NULL score/rank, B<=0, n<=0, k outside [0,n]), UNSUPPORTED (n > 65536;
+ * n > 51200 when kept_idx or near_tie is asked for).
  */
 lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_stride, int k,
                              int32_t* rank, int32_t* kept_idx, int32_t* near_tie,

@@ -95,6 +95,7 @@ extern "C" lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_
     if (score_stride == 0) score_stride = n;
     if (score_stride < n) return LVLM_ERR_INVALID_ARG;
     if (n > kRankMaxKeys) return LVLM_ERR_UNSUPPORTED;
+    if ((kept_idx || near_tie) && (size_t)n * 4 > (size_t)kMaxDynSmem) return LVLM_ERR_UNSUPPORTED;
     int S, slice_len, jt;
     rank_shape(n, B, &S, &slice_len, &jt);
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(select_count_kernel,
