@@ -594,10 +594,16 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
         SimArgs a;
         a.r = L.r; a.k = d->k; a.nkc = (d->C + kSimK - 1) / kSimK; a.nct = (d->k + kSimN - 1) / kSimN;
         const int row_tiles = (L.r + kSimM - 1) / kSimM;
-        int nsplit = (148 + row_tiles * d->B - 1) / (row_tiles * d->B);       // enough CTAs for every SM
-        nsplit = nsplit < 1 ? 1 : (nsplit > a.nct ? a.nct : nsplit);
-        a.cps = (a.nct + nsplit - 1) / nsplit;
-        nsplit = (a.nct + a.cps - 1) / a.cps;
+        // column splits: one CTA per SM at a time, so the kernel takes waves x (column tiles per CTA + a
+        // little for the set-up of a CTA); take the split with the smallest product
+        int nsplit = 1;
+        double best_est = 1e30;
+        for (int ns = 1; ns <= a.nct; ++ns) {
+            const int cps = (a.nct + ns - 1) / ns, used = (a.nct + cps - 1) / cps;
+            const int64_t ctas = (int64_t)row_tiles * d->B * used;
+            const double est = (double)((ctas + 147) / 148) * (cps + 0.25);
+            if (est < best_est - 1e-9) { best_est = est; nsplit = used; a.cps = cps; }
+        }
         a.inv_norm = inv_norm; a.best = best; a.dev_status = dev_status;
         const size_t smem = 1024 + (size_t)kSimStageBytes * kSimStages + sizeof(SimSmem);
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(nk_sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
