@@ -159,7 +159,8 @@ lvlm_status lvlm_select_topk(const float* score, int B, int n, int64_t score_str
  * tensor unchanged.  In mode NEAREST_KEPT there is no P_new row and the result has
  * N-(n-k) rows.
  *   hidden      [B][N][C] bf16 (batch stride d->hid_stride_b)
- *   hidden_out  [B][rows after][C] bf16, or NULL to compact `hidden` in place
+ *   hidden_out  [B][rows after][C] bf16, or NULL (or `hidden` itself) to compact `hidden` in place;
+ *               any other overlap with `hidden` is INVALID_ARG
  *   Kc, Vc      optional [B][Hkv][cap][D] bf16: this layer's keys and values, rows 0..N-1
  *               valid; compacted IN PLACE with the same map, the merged row being the same
  *               weighted mean per KV head (pass both or neither)

@@ -303,7 +303,9 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
                                              beta_ppm, budget, src_map, meta, nout, dev_status);
         if (st != LVLM_OK) return st;
     }
-    return launch_inplace_compact(Kc, Vc, kv_sb * 2, kv_sh * 2, d->B, d->Hkv, kHeadDim / 8, 0,
-                                  src_map, nullptr, meta, d->cap, 0, 0, 0, 1, stream,
-                                  /*maps_per_g=*/d->Hkv, /*map_stride=*/d->cap, nout);
+    CompactJob j;
+    j.base0 = Kc; j.base1 = Vc; j.stride_b = kv_sb * 2; j.stride_g = kv_sh * 2; j.B = d->B; j.G = d->Hkv;
+    j.V = kHeadDim / 8; j.src_map = src_map; j.maps_per_g = d->Hkv; j.map_stride = d->cap;
+    j.meta = meta; j.meta_stride = 1; j.nout = nout; j.N = d->cap;
+    return launch_inplace_compact(j, stream);
 }

@@ -6,38 +6,68 @@
 // every output row, a destination for every input row and a merge weight for every image token;
 // (2) one streaming kernel reads every input row of the hidden states once, moves it if it is
 // kept and adds it to the weighted sum if it is merged; (3) one kernel compacts K and V in place.
+#include <mutex>
+
 #include "common.cuh"
 #include "compact.cuh"
 #include "merge.cuh"
+#include "sm100.cuh"
 
 namespace lvlm {
 
 struct MergeLayout {
-    int r1, r, Nout, V;
+    int r1, r, Nout, V, kvP;
     HiddenGrid grid;
-    size_t off_src, off_dst, off_wgt, off_meta, off_partial, total;
+    size_t off_src, off_dst, off_wgt, off_meta, off_partial, off_kvpartial, total;
 };
 
-constexpr int kHidThreads = 256;       // streaming kernel: thread = 16-byte column group (+256, +512 ...)
+constexpr int kHidThreads = 256;       // consumer threads: thread = 16-byte column group (+256, +512 ...)
+constexpr int kStreamThreads = kHidThreads + 64;   // ... plus the warps that issue the bulk loads and stores
 constexpr int kHidMaxChunks = 4;       // column groups per thread: rows up to 4 * 256 * 8 = 8192 channels
-constexpr int kNoRow = -2147483647 - 1;  // marks a slot of a row group that lies past the last row
+constexpr int kNoRow = -2147483647 - 1;  // marks a slot of a tile that holds no row
 constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
+constexpr int kStreamMaxStages = 16;   // tiles in flight per CTA
+constexpr int kStreamRingBytes = 172 * 1024;  // shared-memory ring of a CTA (one CTA per SM)
+constexpr int kStreamTileBytes = 34 * 1024;   // rows are grouped into tiles of about this size
+constexpr int kKvRowBytes = kHeadDim * 2;
 
-// One wave of CTAs over the whole batch (four per SM fit for rows up to 4096 channels, two beyond:
-// the registers of the row groups in flight decide), at least 8 input rows each; clusters of 8.
+// One CTA per SM over the whole batch, at least two tiles of rows each; the CTAs of a sequence form
+// clusters (their partial sums of the merged row are added through distributed shared memory).
 HiddenGrid hidden_grid(const lvlm_dims* d) {
     HiddenGrid g;
     g.V = d->C / 8;
-    const int per_sm = (g.V + kHidThreads - 1) / kHidThreads <= 2 ? 4 : 2;
-    int cps = (per_sm * 148) / d->B;
-    const int max_by_rows = (d->N + 7) / 8;
-    cps = cps > max_by_rows ? max_by_rows : cps;
-    cps = cps < 1 ? 1 : cps;
-    g.cl = cps >= kHidCluster ? kHidCluster : 1;
-    cps = cps / g.cl * g.cl;
-    g.cps = cps;
-    g.rpc = (d->N + cps - 1) / cps;
+    const int rowB = d->C * 2;
+    int rpt = kStreamTileBytes / rowB;
+    rpt = rpt < 1 ? 1 : (rpt > 32 ? 32 : rpt);
+    g.rpt = rpt;
+    g.slotB = rpt * rowB;
+    if (g.slotB < 16 * kKvRowBytes) g.slotB = 16 * kKvRowBytes;    // room for a tile of K or V rows
+    g.slotB = (g.slotB + 127) / 128 * 128;
+    int ns = kStreamRingBytes / g.slotB;
+    g.nstage = ns > kStreamMaxStages ? kStreamMaxStages : ns;
+    const int tiles = (d->N + rpt - 1) / rpt;
+    int raw = 148 / d->B;
+    raw = raw > tiles / 2 ? tiles / 2 : raw;
+    raw = raw < 1 ? 1 : raw;
+    g.cl = 1; g.cps = 0;
+    for (int cl = kHidCluster; cl >= 1; cl >>= 1) {        // the cluster size that uses the most CTAs, the larger on a tie
+        const int c = raw / cl * cl;
+        if (c >= 1 && c / cl <= 48 && c > g.cps) { g.cps = c; g.cl = cl; }
+    }
+    if (g.cps == 0) { g.cps = raw > 48 ? 48 : raw; g.cl = 1; }
     return g;
+}
+
+// Chunks the image span of every K and V sequence is cut into when the merged rows are summed: about four
+// work items per CTA of the sequence's batch element (the CTAs take them in turn), not shorter than 128 rows.
+static int kv_chunks(const lvlm_dims* d, const HiddenGrid& g) {
+    if (d->Hkv <= 0) return 1;
+    int p = (4 * g.cps + d->Hkv * 2 - 1) / (d->Hkv * 2);
+    const int by_rows = d->n / 128;
+    p = p > by_rows ? by_rows : p;
+    p = p < 1 ? 1 : p;
+    while (p > 1 && (int64_t)(p - 1) * ((d->n + p - 1) / p) >= d->n) --p;      // no chunk is empty
+    return p;
 }
 
 static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
@@ -49,6 +79,7 @@ static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
     L->Nout = d->N - L->r;
     L->V = d->C / 8;
     L->grid = hidden_grid(d);
+    L->kvP = kv_chunks(d, L->grid);
     const int cps = L->grid.cps;
     size_t off = 0;
     L->off_src = off;     off = align_up(off + (size_t)d->B * d->N * 4, 256);
@@ -56,6 +87,8 @@ static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
     L->off_wgt = off;     off = align_up(off + (size_t)d->B * d->n * 4, 256);
     L->off_meta = off;    off = align_up(off + (size_t)d->B * kMetaInts * 4, 256);
     L->off_partial = off; off = align_up(off + (size_t)d->B * (cps / L->grid.cl) * d->C * 4, 256);
+    L->off_kvpartial = off;
+    if (d->Hkv > 0) off = align_up(off + (size_t)d->B * d->Hkv * 2 * L->kvP * kHeadDim * 4, 256);
     L->total = off;
     return true;
 }
@@ -257,30 +290,120 @@ __device__ __forceinline__ float4 hid_ld_cluster_f4(const float* my_smem, uint32
     return v;
 }
 
-// Hidden states, out of place.  grid (CTAs per sequence, B), clusters of `cl` CTAs along x.  A CTA
-// takes every grid.x-th group of two consecutive INPUT rows and reads each row exactly once: a kept
-// row goes to its destination, a merged row is added, times its weight, to fp32 sums the thread
-// keeps for its columns (its rows in increasing order).  The CTAs of a cluster add their sums in rank
-// order through distributed shared memory and park one partial per cluster; the last cluster of
-// the sequence to finish adds the partials in cluster order, rounds once to bf16 and writes P_new.
+// One pass over the rows.  grid (CTAs per sequence, B), clusters of `cl` CTAs along x.  A CTA is eight consumer
+// warps, a loader warp and a storer warp around a ring of shared-memory tiles, each guarded by a "full" mbarrier
+// (bytes landed) and an "empty" mbarrier (every consumer warp and the storer are done with it).  A tile is a run of
+// consecutive rows, fetched by ONE bulk copy (cp.async.bulk; a copy costs the issuing warp about as much whatever
+// its size, so they are made large), so each row is read exactly once.
+//
+// First the tiles of K and V (only with Kc): the image span of every (KV head, K|V) is cut into chunks, a CTA
+// takes every grid.x-th chunk; the consumers add the rows that are merged away, times their weights, in row
+// order, and leave one fp32 partial row per chunk for the compaction kernel, which adds the chunks in order.
+// (Kept rows of these tiles come along unused: fetching 256-byte rows one by one would cost more.)
+//
+// Then the hidden states: tiles of consecutive INPUT rows are dealt round robin, so that every CTA gets the same
+// mix of kept rows (read and written) and merged rows (read only).  Kept rows leave again by bulk copies from
+// shared memory to their destination (the storer issues one per run of rows whose destinations are contiguous; no
+// register ever holds a row), merged rows are added by the consumers to fp32 sums each thread keeps for its columns
+// (its rows in increasing order).  The CTAs of a cluster add their sums in rank order through distributed shared
+// memory, each a slice of the columns, and park one partial per cluster; the compaction launch that follows adds
+// the partials in cluster order, rounds once to bf16 and writes P_new.
+// Without `out` nothing is stored: only merged rows are read.
+//
+// Destination and weight of every row of a tile travel beside it: the loader copies them (cp.async, 4 bytes each)
+// into a table a dozen tiles ahead, so that nobody ever waits for them.
+struct StreamArgs {
+    const char* hid; char* out; char* scratch;
+    int64_t hid_sb, out_sb, scr_sb;                      // bytes
+    int rowB, V, N, i0, n, k, cl, rpt, slotB, nstage;
+    const int32_t* dst_map; const float* wgt; int32_t* meta; float* partial;
+    const char* K; const char* Vc; int64_t kv_sb, kv_sh; // bytes
+    int Hkv, kvP, kvL, kvT;
+    float* kv_partial;
+    int32_t* dev_status;
+};
+
+constexpr int kTabTiles = 32;          // tiles whose row tables are held at a time
+constexpr int kTabAhead = 12;          // ... and how far ahead of the tile being fetched they are requested
+constexpr int kTabRows = 64;           // most rows a tile can hold
+constexpr int kLoaderWarp = kHidThreads / 32, kStorerWarp = kLoaderWarp + 1;
+
+__device__ __forceinline__ void cp_async4(void* smem, const void* gmem) {
+    const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(sa), "l"(gmem) : "memory");
+}
+
 template <int CH>
-__global__ void __launch_bounds__(kHidThreads, CH <= 2 ? 4 : 2)     // the occupancy hidden_grid() counts on
-hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
-                     int64_t hid_stride_b, int64_t out_stride_b,   // in uint4
-                     int V, int N, int i0, int n, int k, int rpc, int cl,
-                     const int32_t* __restrict__ dst_map, const float* __restrict__ wgt,
-                     int32_t* meta, float* partial, uint4* __restrict__ scratch, int64_t scr_stride_b) {
-    extern __shared__ __align__(16) float s_sum[];           // [V][8] this CTA's sums
-    __shared__ int s_last;
-    pdl_enter();
-    const int b = blockIdx.y, cta = blockIdx.x, tid = threadIdx.x;
-    const uint4* hin = hidden + (int64_t)b * hid_stride_b;
-    uint4* hout = out + (int64_t)b * out_stride_b;
-    const int32_t* dst = dst_map + (int64_t)b * N;
-    const float* w = wgt ? wgt + (int64_t)b * n - i0 : nullptr;   // indexed by sequence position
-    uint4* scr = scratch ? scratch + (int64_t)b * scr_stride_b : nullptr;
-    const int i_hi = N;
-    (void)rpc;
+__global__ void __launch_bounds__(kStreamThreads, 1) row_stream_kernel(const StreamArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) uint64_t s_full[kStreamMaxStages];
+    __shared__ __align__(8) uint64_t s_empty[kStreamMaxStages];
+    __shared__ __align__(8) uint64_t s_tab_ready;           // the tables of the tiles fetched before the wait are in place
+    __shared__ int s_tab_d[kTabTiles][kTabRows];            // destination and weight of the rows of a tile
+    __shared__ float s_tab_w[kTabTiles][kTabRows];
+    __shared__ __align__(16) float s_red[16 * kHeadDim];
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.y, cta = blockIdx.x, cps = (int)gridDim.x;
+    const int S = a.nstage;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { sm100::mbar_init(&s_full[s], 1); sm100::mbar_init(&s_empty[s], kHidThreads / 32 + 1); }
+        sm100::mbar_init(&s_tab_ready, 1);
+        s_abort = 0;
+        sm100::fence_barrier_init();
+    }
+    __syncthreads();
+    // The kernel ahead in the stream (the plan) writes the row maps and weights only, and it has itself waited for
+    // everything before it: the rows can be fetched while it still runs.  The loader does so for the first lap of
+    // the ring before it waits; every other warp waits here.
+    if (warp != kLoaderWarp) pdl_wait();
+    pdl_launch_dependents();
+
+    const int32_t* dst = a.dst_map + (int64_t)b * a.N;
+    const float* w = a.wgt ? a.wgt + (int64_t)b * a.n - a.i0 : nullptr;     // indexed by sequence position
+    // My tiles: first those of my K/V chunks, then those of the hidden states.  Every role walks them with its own
+    // iterator (the loader with two: one runs ahead for the row tables); no division outside the start of a chunk.
+    const int nItems = a.K ? a.Hkv * 2 * a.kvP : 0;
+    struct Tile { int first, cnt, kv, item_end, item; const char* from; };
+    struct TileIt {
+        const StreamArgs& a; int b, cta, cps, nItems;
+        int item, tb, r1, row; const char* seq;
+        __device__ TileIt(const StreamArgs& a_, int b_, int cta_, int cps_, int nItems_)
+            : a(a_), b(b_), cta(cta_), cps(cps_), nItems(nItems_), item(cta_ - cps_), tb(0), r1(0), row(cta_ * a_.rpt), seq(nullptr) {}
+        __device__ bool next(Tile* t) {
+            while (item < nItems) {
+                if (tb < r1) {
+                    t->first = tb; t->cnt = min(a.kvT, r1 - tb); t->kv = 1; t->item = item;
+                    t->from = seq + (int64_t)tb * kKvRowBytes;
+                    tb += a.kvT;
+                    t->item_end = tb >= r1;
+                    return true;
+                }
+                item += cps;
+                if (item < nItems) {
+                    const int chunk = item % a.kvP, gw = item / a.kvP;
+                    tb = a.i0 + chunk * a.kvL;
+                    r1 = min(a.i0 + a.n, tb + a.kvL);
+                    seq = ((gw & 1) ? a.Vc : a.K) + (int64_t)b * a.kv_sb + (int64_t)(gw >> 1) * a.kv_sh;
+                }
+            }
+            if (row < a.N) {
+                t->first = row; t->cnt = min(a.rpt, a.N - row); t->kv = 0; t->item_end = 0; t->item = 0;
+                t->from = a.hid + (int64_t)b * a.hid_sb + (int64_t)row * a.rowB;
+                row += cps * a.rpt;
+                return true;
+            }
+            return false;
+        }
+    };
+    volatile int* abort_flag = &s_abort;
+    auto wait_on = [&](uint64_t* bar, uint32_t parity) -> bool {
+        if (sm100::mbar_wait(bar, parity)) return true;
+        *abort_flag = 1;
+        if (a.dev_status) atomicOr(a.dev_status, LVLM_DEV_TIMEOUT);
+        return false;
+    };
 
     float acc[CH][8];
 #pragma unroll
@@ -288,183 +411,297 @@ hidden_stream_kernel(const uint4* __restrict__ hidden, uint4* __restrict__ out,
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[ci][e] = 0.f;
 
-    // Groups of kG rows are dealt out round robin, so that every CTA gets the same mix of kept rows (read
-    // and written) and merged rows (read only).  Two groups are in flight in turn: the loads of the next
-    // one are issued before the current one is used.
-    constexpr int kG = 2;
-    auto load_group = [&](int ib, int* d, float* wj, uint4 (*x)[CH]) {
-#pragma unroll
-        for (int u = 0; u < kG; ++u) {
-            const int i = ib + u;
-            d[u] = i < i_hi ? dst[i] : kNoRow;
-            wj[u] = (w && i < i_hi && i >= i0 && i < i0 + n) ? w[i] : 0.f;
-#pragma unroll
-            for (int ci = 0; ci < CH; ++ci) {
-                const int c = tid + ci * kHidThreads;
-                x[u][ci] = (i < i_hi && c < V) ? __ldg(hin + (int64_t)i * V + c) : make_uint4(0, 0, 0, 0);
-            }
-        }
-    };
-    auto use_group = [&](const int* d, const float* wj, const uint4 (*x)[CH]) {
-#pragma unroll
-        for (int u = 0; u < kG; ++u) {
-            if (d[u] >= 0) {
-#pragma unroll
-                for (int ci = 0; ci < CH; ++ci) {
-                    const int c = tid + ci * kHidThreads;
-                    if (c < V) hout[(int64_t)d[u] * V + c] = x[u][ci];
+    if (warp == kLoaderWarp) {
+        // ---- loader ----------------------------------------------------------------------------------------
+        TileIt ahead(a, b, cta, cps, nItems), it(a, b, cta, cps, nItems);
+        int ja = 0;                                         // tiles whose tables have been requested
+        auto request_table = [&]() {                        // destination and weight of the rows of the next tile ahead
+            Tile t;
+            if (ahead.next(&t)) {
+                int* td = s_tab_d[ja & (kTabTiles - 1)];
+                float* tw = s_tab_w[ja & (kTabTiles - 1)];
+                for (int e = lane; e < t.cnt; e += 32) {
+                    const int i = t.first + e;
+                    cp_async4(&td[e], dst + i);
+                    if (w && i >= a.i0 && i < a.i0 + a.n) cp_async4(&tw[e], w + i);
                 }
-            } else if (d[u] <= -2 && d[u] != kNoRow) {        // a row set aside: scratch row -d-2
-                if (scr) {
+            }
+            ++ja;
+            asm volatile("cp.async.commit_group;\n" ::: "memory");
+        };
+        auto fetch = [&](const Tile& t, int slot, int j) {
+            unsigned char* sbase = ring + (size_t)slot * a.slotB;
+            const uint32_t rb = t.kv ? (uint32_t)kKvRowBytes : (uint32_t)a.rowB;
+            if (t.kv || a.out) {                            // the whole tile in one copy
+                if (lane == 0) {
+                    sm100::mbar_arrive_expect_tx(&s_full[slot], (uint32_t)t.cnt * rb);
+                    sm100::bulk_load(sbase, t.from, (uint32_t)t.cnt * rb, &s_full[slot]);
+                }
+            } else {                                        // merged rows only (cnt <= 32 here)
+                const bool need = lane < t.cnt && s_tab_d[j & (kTabTiles - 1)][lane] == -1;
+                const unsigned bal = __ballot_sync(0xFFFFFFFFu, need);
+                if (lane == 0) sm100::mbar_arrive_expect_tx(&s_full[slot], (uint32_t)__popc(bal) * rb);
+                __syncwarp();
+                if (need) sm100::bulk_load(sbase + (size_t)lane * rb, t.from + (int64_t)lane * rb, rb, &s_full[slot]);
+            }
+        };
+        Tile t;
+        int slot = 0, j = 0;
+        bool more = it.next(&t);
+        // whole-tile copies need no table: the first lap of the ring starts before the wait
+        for (; more && j < S && (t.kv || a.out); ++j, ++slot) { fetch(t, slot, j); more = it.next(&t); }
+        pdl_wait();
+        for (int q = 0; q < j + kTabAhead; ++q) request_table();
+        asm volatile("cp.async.wait_group %0;\n" ::"n"(kTabAhead) : "memory");          // the tables of the tiles under way
+        __syncwarp();
+        if (lane == 0) sm100::mbar_arrive(&s_tab_ready);
+        uint32_t phase = 0;                                 // parity of the "empty" phase awaited; no wait in the first lap
+        bool ok = true, first_lap = true;
+        if (slot == S) { slot = 0; first_lap = false; }
+        while (more) {
+            request_table();
+            if (!first_lap && ok) ok = wait_on(&s_empty[slot], phase);                // everybody is done with the slot
+            asm volatile("cp.async.wait_group %0;\n" ::"n"(kTabAhead) : "memory");      // the table of this tile is in place
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (ok) fetch(t, slot, j);
+            ++j;
+            if (++slot == S) { slot = 0; if (first_lap) first_lap = false; else phase ^= 1u; }
+            more = it.next(&t);
+        }
+        asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    } else if (warp == kStorerWarp) {
+        // ---- storer: lane l owns row l of a tile -------------------------------------------------------------
+        TileIt it(a, b, cta, cps, nItems);
+        Tile t;
+        int slot = 0, j = 0, prev_slot = -1;
+        uint32_t phase = 0;
+        bool ok = wait_on(&s_tab_ready, 0);
+        while (it.next(&t)) {
+            if (ok) ok = wait_on(&s_full[slot], phase);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (ok && !t.kv && a.out) {                     // the kept rows leave again
+                const int dd = lane < t.cnt ? s_tab_d[j & (kTabTiles - 1)][lane] : kNoRow;
+                char* to = nullptr;
+                if (dd >= 0) to = a.out + (int64_t)b * a.out_sb + (int64_t)dd * a.rowB;
+                else if (dd <= -2 && dd != kNoRow && a.scratch)       // a row set aside: scratch row -d-2
+                    to = a.scratch + (int64_t)b * a.scr_sb + (int64_t)(-dd - 2) * a.rowB;
+                // runs of rows whose destinations follow each other leave in one copy, issued by the run's first lane
+                const unsigned long long toi = (unsigned long long)to;
+                const unsigned long long prev = __shfl_up_sync(0xFFFFFFFFu, toi, 1);
+                const bool head = to != nullptr && (lane == 0 || prev == 0ull || prev + (unsigned long long)a.rowB != toi);
+                const unsigned heads = __ballot_sync(0xFFFFFFFFu, head);
+                const unsigned valid = __ballot_sync(0xFFFFFFFFu, to != nullptr);
+                if (head) {
+                    const unsigned above = lane == 31 ? 0u : (~0u << (lane + 1));
+                    const unsigned stop = (heads | ~valid) & above;              // the next head, or the next row that stays
+                    const int end = stop ? __ffs(stop) - 1 : 32;
+                    sm100::bulk_store(to, ring + (size_t)slot * a.slotB + (size_t)lane * a.rowB,
+                                      (uint32_t)(end - lane) * (uint32_t)a.rowB);
+                }
+            }
+            sm100::bulk_commit();                           // one group per tile, empty or not
+            if (prev_slot >= 0) {
+                sm100::bulk_wait_read<1>();                 // the stores of the tile before have left its slot
+                __syncwarp();
+                if (lane == 0) sm100::mbar_arrive(&s_empty[prev_slot]);
+            }
+            prev_slot = slot;
+            ++j;
+            if (++slot == S) { slot = 0; phase ^= 1u; }
+        }
+        sm100::bulk_wait<0>();
+    } else {
+        // ---- consumers -----------------------------------------------------------------------------------
+        const int rl = tid >> 4, cg = tid & 15;             // K/V tiles: row lane and 16-byte column group
+        float kacc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        TileIt it(a, b, cta, cps, nItems);
+        Tile t;
+        int slot = 0, j = 0;
+        uint32_t phase = 0;
+        bool ok = wait_on(&s_tab_ready, 0);
+        while (it.next(&t)) {
+            const unsigned char* sbase = ring + (size_t)slot * a.slotB;
+            const int* td = s_tab_d[j & (kTabTiles - 1)];
+            const float* tw = s_tab_w[j & (kTabTiles - 1)];
+            if (ok) ok = wait_on(&s_full[slot], phase);
+            if (ok && t.kv) {
+                for (int p = rl; p < t.cnt; p += 16) {
+                    if (td[p] != -1) continue;
+                    const float wj = tw[p];
+                    const uint4 xv = *reinterpret_cast<const uint4*>(sbase + p * kKvRowBytes + cg * 16);
+                    kacc[0] = fmaf(wj, bf16_lo(xv.x), kacc[0]); kacc[1] = fmaf(wj, bf16_hi(xv.x), kacc[1]);
+                    kacc[2] = fmaf(wj, bf16_lo(xv.y), kacc[2]); kacc[3] = fmaf(wj, bf16_hi(xv.y), kacc[3]);
+                    kacc[4] = fmaf(wj, bf16_lo(xv.z), kacc[4]); kacc[5] = fmaf(wj, bf16_hi(xv.z), kacc[5]);
+                    kacc[6] = fmaf(wj, bf16_lo(xv.w), kacc[6]); kacc[7] = fmaf(wj, bf16_hi(xv.w), kacc[7]);
+                }
+            } else if (ok && w) {
+                for (int l = 0; l < t.cnt; ++l) {
+                    if (td[l] != -1) continue;
+                    const float wj = tw[l];
+                    const uint4* rowp = reinterpret_cast<const uint4*>(sbase + (size_t)l * a.rowB);
 #pragma unroll
                     for (int ci = 0; ci < CH; ++ci) {
                         const int c = tid + ci * kHidThreads;
-                        if (c < V) scr[(int64_t)(-d[u] - 2) * V + c] = x[u][ci];
+                        if (c < a.V) {
+                            const uint4 xv = rowp[c];
+                            acc[ci][0] = fmaf(wj, bf16_lo(xv.x), acc[ci][0]); acc[ci][1] = fmaf(wj, bf16_hi(xv.x), acc[ci][1]);
+                            acc[ci][2] = fmaf(wj, bf16_lo(xv.y), acc[ci][2]); acc[ci][3] = fmaf(wj, bf16_hi(xv.y), acc[ci][3]);
+                            acc[ci][4] = fmaf(wj, bf16_lo(xv.z), acc[ci][4]); acc[ci][5] = fmaf(wj, bf16_hi(xv.z), acc[ci][5]);
+                            acc[ci][6] = fmaf(wj, bf16_lo(xv.w), acc[ci][6]); acc[ci][7] = fmaf(wj, bf16_hi(xv.w), acc[ci][7]);
+                        }
                     }
                 }
-            } else if (d[u] == -1) {
-#pragma unroll
-                for (int ci = 0; ci < CH; ++ci) {
-                    acc[ci][0] = fmaf(wj[u], bf16_lo(x[u][ci].x), acc[ci][0]); acc[ci][1] = fmaf(wj[u], bf16_hi(x[u][ci].x), acc[ci][1]);
-                    acc[ci][2] = fmaf(wj[u], bf16_lo(x[u][ci].y), acc[ci][2]); acc[ci][3] = fmaf(wj[u], bf16_hi(x[u][ci].y), acc[ci][3]);
-                    acc[ci][4] = fmaf(wj[u], bf16_lo(x[u][ci].z), acc[ci][4]); acc[ci][5] = fmaf(wj[u], bf16_hi(x[u][ci].z), acc[ci][5]);
-                    acc[ci][6] = fmaf(wj[u], bf16_lo(x[u][ci].w), acc[ci][6]); acc[ci][7] = fmaf(wj[u], bf16_hi(x[u][ci].w), acc[ci][7]);
-                }
             }
-        }
-    };
-    {
-        const int step = (int)gridDim.x * kG;
-        int dA[kG], dB[kG];
-        float wA[kG], wB[kG];
-        uint4 xA[kG][CH], xB[kG][CH];
-        int ib = cta * kG;
-        load_group(ib, dA, wA, xA);
-        for (; ib < i_hi; ib += 2 * step) {
-            load_group(ib + step, dB, wB, xB);
-            use_group(dA, wA, xA);
-            load_group(ib + 2 * step, dA, wA, xA);
-            use_group(dB, wB, xB);
-        }
-    }
-
-    if (!w) return;                                           // no merged row in this mode
-    // ---- clusters that touch the image span contribute a partial sum ---------------------------------
-    const int cluster = cta / cl;
-    const int q_first = 0, q_last = (int)gridDim.x / cl - 1;  // every cluster has seen merged rows
-    const int rank = (int)hid_cluster_rank();
+            __syncwarp();
+            if (lane == 0) sm100::mbar_arrive(&s_empty[slot]);
+            if (t.kv && t.item_end) {
+                // end of a chunk: row lanes added in lane order, one partial row parked for the compaction kernel
 #pragma unroll
-    for (int ci = 0; ci < CH; ++ci) {
-        const int c = tid + ci * kHidThreads;
-        if (c < V) {
-            *reinterpret_cast<float4*>(s_sum + c * 8) = make_float4(acc[ci][0], acc[ci][1], acc[ci][2], acc[ci][3]);
-            *reinterpret_cast<float4*>(s_sum + c * 8 + 4) = make_float4(acc[ci][4], acc[ci][5], acc[ci][6], acc[ci][7]);
+                for (int e = 0; e < 8; ++e) { s_red[(rl * 16 + cg) * 8 + e] = kacc[e]; kacc[e] = 0.f; }
+                asm volatile("bar.sync 1, %0;" ::"n"(kHidThreads) : "memory");
+                if (tid < kHeadDim) {
+                    float r = 0.f;
+#pragma unroll
+                    for (int l = 0; l < 16; ++l) r += s_red[l * kHeadDim + tid];
+                    a.kv_partial[((int64_t)b * nItems + t.item) * kHeadDim + tid] = r;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kHidThreads) : "memory");
+            }
+            ++j;
+            if (++slot == S) { slot = 0; phase ^= 1u; }
         }
     }
-    hid_cluster_barrier();
-    if (rank == 0) {
-        float* my_partial = partial + ((int64_t)b * gridDim.x / cl + cluster) * V * 8;
+    __syncthreads();
+    if (s_abort) {                                             // copies may still be in flight: let them land
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (!w) return;                                            // no merged row in this mode
+
+    // ---- the merged row of the hidden states --------------------------------------------------------------
+    float* s_sum = reinterpret_cast<float*>(ring);            // [V][8] this CTA's sums; the ring is free now
+    const int V = a.V, cl = a.cl;
+    const int cluster = cta / cl;
+    const int nq = cps / cl;                                   // partials of this sequence, one per cluster
+    const int rank = (int)hid_cluster_rank();
+    if (tid < kHidThreads) {
 #pragma unroll
         for (int ci = 0; ci < CH; ++ci) {
             const int c = tid + ci * kHidThreads;
             if (c < V) {
-                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-                for (int r = 0; r < cl; ++r) {
-                    const float4 a0 = hid_ld_cluster_f4(s_sum + c * 8, r), a1 = hid_ld_cluster_f4(s_sum + c * 8 + 4, r);
-                    lo.x += a0.x; lo.y += a0.y; lo.z += a0.z; lo.w += a0.w;
-                    hi.x += a1.x; hi.y += a1.y; hi.z += a1.z; hi.w += a1.w;
-                }
-                *reinterpret_cast<float4*>(my_partial + c * 8) = lo;
-                *reinterpret_cast<float4*>(my_partial + c * 8 + 4) = hi;
+                *reinterpret_cast<float4*>(s_sum + c * 8) = make_float4(acc[ci][0], acc[ci][1], acc[ci][2], acc[ci][3]);
+                *reinterpret_cast<float4*>(s_sum + c * 8 + 4) = make_float4(acc[ci][4], acc[ci][5], acc[ci][6], acc[ci][7]);
             }
         }
     }
-    // ---- the last cluster of this sequence finalises P_new, all of its CTAs sharing the columns -----------
-    if (rank == 0) {
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            const int ticket = atomicAdd(&meta[b * kMetaInts + 1], 1);
-            s_last = ticket == q_last - q_first;
-        }
-    }
-    hid_cluster_barrier();                 // rank 0 has read every CTA's sums and knows whether we are last
-    const int last = cl > 1 ? hid_ld_cluster_i32(&s_last, 0) : s_last;
-    hid_cluster_barrier();                 // ... and everybody has asked it
-    if (!last) return;
-    __threadfence();
-    const int nq = q_last - q_first + 1;                      // partials to add, in cluster order
+    hid_cluster_barrier();
     const int Vs = (V + cl - 1) / cl;                         // my slice of the column groups
     const int c_lo = min(V, rank * Vs), c_hi = min(V, c_lo + Vs);
-    // two threads per column group, each adding half of the partials (four in flight); the halves are
-    // added in order through shared memory
-    const int hsel = tid >> 7, lane_c = tid & 127;
-    const int q_mid = q_first + (nq + 1) / 2;
-    const int qa = hsel ? q_mid : q_first, qb = hsel ? q_last + 1 : q_mid;
-    float* s_fin = s_sum;                                     // [2][c_hi - c_lo][8], free after the barriers
-    for (int cb = c_lo; cb < c_hi; cb += 128) {
-        const int c = cb + lane_c;
-        float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        if (c < c_hi) {
-            for (int q = qa; q < qb; q += 4) {
-                float4 lo[4], hi[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    lo[u] = hi[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (q + u < qb) {
-                        const float4* pp = reinterpret_cast<const float4*>(
-                            partial + ((int64_t)b * gridDim.x / cl + q + u) * V * 8 + c * 8);
-                        lo[u] = __ldcg(pp); hi[u] = __ldcg(pp + 1);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    t[0] += lo[u].x; t[1] += lo[u].y; t[2] += lo[u].z; t[3] += lo[u].w;
-                    t[4] += hi[u].x; t[5] += hi[u].y; t[6] += hi[u].z; t[7] += hi[u].w;
-                }
+    {
+        // every CTA adds its slice of the columns over the CTAs of the cluster, in rank order
+        float* my_partial = a.partial + ((int64_t)b * nq + cluster) * V * 8;
+        for (int idx = tid; idx < (c_hi - c_lo) * 2; idx += kStreamThreads) {
+            const int c = c_lo + (idx >> 1), half = idx & 1;
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r = 0; r < cl; ++r) {
+                const float4 x = hid_ld_cluster_f4(s_sum + c * 8 + half * 4, r);
+                t.x += x.x; t.y += x.y; t.z += x.z; t.w += x.w;
             }
-#pragma unroll
-            for (int e = 0; e < 8; ++e) s_fin[(hsel * Vs + (c - c_lo)) * 8 + e] = t[e];
+            *reinterpret_cast<float4*>(my_partial + c * 8 + half * 4) = t;
         }
     }
-    __syncthreads();
-    for (int c = c_lo + tid; c < c_hi; c += kHidThreads) {
-        float t[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) t[e] = s_fin[(c - c_lo) * 8 + e] + s_fin[(Vs + (c - c_lo)) * 8 + e];
-        uint4 o;
-        o.x = pack_bf16(t[0], t[1]); o.y = pack_bf16(t[2], t[3]);
-        o.z = pack_bf16(t[4], t[5]); o.w = pack_bf16(t[6], t[7]);
-        hout[(int64_t)(i0 + k) * V + c] = o;
-    }
-    if (rank == 0 && tid == 0) meta[b * kMetaInts + 1] = 0;
+    hid_cluster_barrier();                 // every CTA's sums have been read: nobody leaves before
 }
 
+// Dynamic shared memory of the streaming kernel: always the whole ring budget, so that how many clusters fit on
+// the GPU depends on the cluster size alone.
+constexpr size_t kStreamSmem = (size_t)kStreamRingBytes;
+
 template <int CH>
-static lvlm_status launch_hidden_stream(const void* hidden, void* hidden_out, int64_t hid_sb, int64_t out_sb,
-                                        const lvlm_dims* d, const HiddenGrid& L, const int32_t* dst_map,
-                                        const float* wgt, int32_t* meta, float* partial, void* scratch,
-                                        int64_t scr_sb, cudaStream_t stream) {
-    const size_t smem = (size_t)L.V * 32 * (L.cl > 1 ? 1 : 2);      // the final sum needs two rows without a cluster
-    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(hidden_stream_kernel<CH>,
+static lvlm_status launch_row_stream(const StreamArgs& a, int cps, int cl, int B, cudaStream_t stream) {
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(row_stream_kernel<CH>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    return launch_kernel(hidden_stream_kernel<CH>, dim3((unsigned)L.cps, (unsigned)d->B), dim3(kHidThreads), smem,
-                         stream, L.cl, static_cast<const uint4*>(hidden), static_cast<uint4*>(hidden_out),
-                         hid_sb / 8, out_sb / 8, L.V, d->N, d->i0, d->n, d->k, L.rpc, L.cl, dst_map, wgt, meta,
-                         partial, static_cast<uint4*>(scratch), scr_sb / 8);
+    return launch_kernel(row_stream_kernel<CH>, dim3((unsigned)cps, (unsigned)B), dim3(kStreamThreads), kStreamSmem,
+                         stream, cl, a);
+}
+
+// How many clusters of `cl` CTAs of the streaming kernel the current device runs at a time (clusters are placed
+// inside one GPC, so fewer CTAs fit than there are SMs); looked up once per device and cluster size.
+template <int CH>
+static int stream_clusters_resident(int cl) {
+    static std::mutex mu;
+    static int cache[64][4];                                // [device][log2 cl], 0 = not looked up yet
+    int dev = 0, lg = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    while ((1 << lg) < cl) ++lg;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache[dev][lg] == 0) {
+        if (cudaFuncSetAttribute(row_stream_kernel<CH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
+            cudaSuccess)
+            return 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(cl * 64));
+        cfg.blockDim = dim3(kStreamThreads);
+        cfg.dynamicSmemBytes = kStreamSmem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, row_stream_kernel<CH>, &cfg) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = 128 / cl;                                   // a safe guess
+        }
+        cache[dev][lg] = n;
+    }
+    return cache[dev][lg];
 }
 
 lvlm_status launch_hidden_rows(const void* hidden, void* hidden_out, int64_t hid_sb, int64_t out_sb,
                                const lvlm_dims* d, const HiddenGrid& L, const int32_t* dst_map,
                                const float* wgt, int32_t* meta, float* partial, void* scratch,
-                               int64_t scr_sb, cudaStream_t stream) {
+                               int64_t scr_sb, cudaStream_t stream, const StreamKv* kv, int32_t* dev_status,
+                               int* partials_out) {
     const int chunks = (L.V + kHidThreads - 1) / kHidThreads;
-    if (chunks > kHidMaxChunks) return LVLM_ERR_UNSUPPORTED;  // more than 8192 channels
+    if (chunks > kHidMaxChunks || L.nstage < 3) return LVLM_ERR_UNSUPPORTED;  // more than 8192 channels
+    // no more clusters than the device runs at a time: a second wave would double the time
+    int resident = 0;
     switch (chunks) {
-        case 1: return launch_hidden_stream<1>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
-        case 2: return launch_hidden_stream<2>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
-        case 3: return launch_hidden_stream<3>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
-        case 4: return launch_hidden_stream<4>(hidden, hidden_out, hid_sb, out_sb, d, L, dst_map, wgt, meta, partial, scratch, scr_sb, stream);
+        case 1: resident = stream_clusters_resident<1>(L.cl); break;
+        case 2: resident = stream_clusters_resident<2>(L.cl); break;
+        case 3: resident = stream_clusters_resident<3>(L.cl); break;
+        case 4: resident = stream_clusters_resident<4>(L.cl); break;
+    }
+    int cps = L.cps;
+    if (resident > 0) {
+        int per_seq = resident / d->B;
+        per_seq = per_seq < 1 ? 1 : per_seq;
+        if (cps > per_seq * L.cl) cps = per_seq * L.cl;
+    }
+    if (partials_out) *partials_out = cps / L.cl;
+    StreamArgs a;
+    a.hid = static_cast<const char*>(hidden);
+    a.out = static_cast<char*>(hidden_out);
+    a.scratch = static_cast<char*>(scratch);
+    a.hid_sb = hid_sb * 2; a.out_sb = out_sb * 2; a.scr_sb = scr_sb * 2;
+    a.rowB = d->C * 2; a.V = L.V; a.N = d->N; a.i0 = d->i0; a.n = d->n; a.k = d->k; a.cl = L.cl;
+    a.rpt = L.rpt; a.slotB = L.slotB; a.nstage = L.nstage;
+    a.dst_map = dst_map; a.wgt = wgt; a.meta = meta; a.partial = partial;
+    a.K = nullptr; a.Vc = nullptr; a.kv_sb = a.kv_sh = 0; a.Hkv = 0; a.kvP = 1; a.kvL = 1; a.kvT = 16;
+    a.kv_partial = nullptr;
+    if (kv && kv->K && wgt) {
+        a.K = static_cast<const char*>(kv->K); a.Vc = static_cast<const char*>(kv->V);
+        a.kv_sb = kv->kv_sb * 2; a.kv_sh = kv->kv_sh * 2; a.Hkv = kv->Hkv; a.kvP = kv->kvP;
+        a.kvL = (d->n + kv->kvP - 1) / kv->kvP;
+        a.kvT = L.slotB / kKvRowBytes >= 64 ? 64 : (L.slotB / kKvRowBytes) / 16 * 16;
+        a.kv_partial = kv->kv_partial;
+    }
+    a.dev_status = dev_status;
+    switch (chunks) {
+        case 1: return launch_row_stream<1>(a, cps, L.cl, d->B, stream);
+        case 2: return launch_row_stream<2>(a, cps, L.cl, d->B, stream);
+        case 3: return launch_row_stream<3>(a, cps, L.cl, d->B, stream);
+        case 4: return launch_row_stream<4>(a, cps, L.cl, d->B, stream);
     }
     return LVLM_ERR_UNSUPPORTED;
 }
@@ -494,6 +731,7 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
         L.Nout = d->N - L.r;
     }
     const int64_t hid_sb = d->hid_stride_b ? d->hid_stride_b : (int64_t)d->N * d->C;
+    if (hidden_out == hidden && mode != LVLM_W_NEAREST_KEPT) hidden_out = nullptr;   // the same buffer: compact in place
     const int64_t out_sb = hidden_out ? (d->out_stride_b ? d->out_stride_b : (int64_t)L.Nout * d->C) : hid_sb;
     const int64_t kv_sh = d->kv_stride_h ? d->kv_stride_h : (int64_t)d->cap * d->D;
     const int64_t kv_sb = d->kv_stride_b ? d->kv_stride_b : (int64_t)d->Hkv * kv_sh;
@@ -501,6 +739,13 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
         hid_sb % 8 || out_sb % 8 || kv_sh % 8 || kv_sb % 8)
         return LVLM_ERR_ALIGNMENT;
     if (hid_sb < (int64_t)d->N * d->C || out_sb < (int64_t)L.Nout * d->C) return LVLM_ERR_INVALID_ARG;
+    if (hidden_out) {     // a separate output must not overlap the input: rows are read and written in no fixed order
+        const char* in0 = static_cast<const char*>(hidden);
+        const char* in1 = in0 + ((int64_t)(d->B - 1) * hid_sb + (int64_t)d->N * d->C) * 2;
+        const char* out0 = static_cast<const char*>(hidden_out);
+        const char* out1 = out0 + ((int64_t)(d->B - 1) * out_sb + (int64_t)L.Nout * d->C) * 2;
+        if (out0 < in1 && in0 < out1) return LVLM_ERR_INVALID_ARG;
+    }
 
     if (L.r <= 0) {                       // keep 100 %: every tensor stays as it is
         if (hidden_out && hidden_out != hidden) {
@@ -528,7 +773,7 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
     else if (mode == LVLM_W_UNIFORM) inv_sum = (float)(1.0 / (double)L.r1);
     const int plan_threads = d->n >= 1024 ? 1024 : (d->n <= 128 ? 128 : ((d->n + 31) / 32) * 32);
     {
-        int P = (d->n + 4095) / 4096;                    // CTAs per sequence: about four tiles of tokens each
+        int P = (d->n + 2047) / 2048;                    // CTAs per sequence: about two tiles of tokens each
         P = P < 1 ? 1 : (P > 8 ? 8 : P);
         const lvlm_status st = launch_kernel(merge_plan_kernel, dim3(P, d->B), dim3(plan_threads), 0, stream, P,
                                              rank, pos_ids, d->N, d->i0, d->n, d->k, (int)mode, inv_sum, w_custom,
@@ -536,20 +781,41 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
         if (st != LVLM_OK) return st;
     }
 
-    if (hidden_out) {
+    float* kv_partial = reinterpret_cast<float*>(wsb + L.off_kvpartial);
+    StreamKv kv = {Kc, Vc, kv_sb, kv_sh, d->Hkv, L.kvP, kv_partial};
+    int hid_partials = L.grid.cps / L.grid.cl;
+    {
+        // one pass over the rows: kept hidden rows to their place (out of place only), merged rows of the hidden
+        // states and of K and V into fp32 sums
         const lvlm_status st = launch_hidden_rows(hidden, hidden_out, hid_sb, out_sb, d, L.grid, dst_map, wgt, meta,
-                                                  partial, nullptr, 0, stream);
-        if (st != LVLM_OK) return st;
-    } else {
-        lvlm_status st = launch_inplace_compact(hidden, nullptr, hid_sb * 2, 0, d->B, 1, L.V,
-                                                L.Nout, src_map, wgt, meta, d->N, d->n, d->i0,
-                                                d->i0 + d->k, kMetaInts, stream, 1, -1, nullptr, dst_map);
+                                                  partial, nullptr, 0, stream, Kc ? &kv : nullptr, dev_status,
+                                                  &hid_partials);
         if (st != LVLM_OK) return st;
     }
+    // P_new of the hidden states: the partial rows are added by the compaction launch that follows
+    if (!hidden_out) {
+        CompactJob j;
+        j.base0 = hidden; j.stride_b = hid_sb * 2; j.B = d->B; j.G = 1; j.V = L.V;
+        j.src_map = src_map; j.map_stride = d->N; j.meta = meta; j.meta_stride = kMetaInts;
+        j.Nout = L.Nout; j.N = d->N; j.merged_row = d->i0 + d->k; j.partial = partial;
+        j.P = hid_partials;
+        const lvlm_status st = launch_inplace_compact(j, stream);
+        if (st != LVLM_OK) return st;
+    }
+    CompactJob j;
+    if (hidden_out) {
+        j.fin_base = hidden_out; j.fin_stride_b = out_sb * 2; j.fin_row = d->i0 + d->k; j.fin_V = L.V;
+        j.fin_partial = partial; j.fin_P = hid_partials;
+    }
     if (Kc) {
-        lvlm_status st = launch_inplace_compact(Kc, Vc, kv_sb * 2, kv_sh * 2, d->B, d->Hkv,
-                                                kHeadDim / 8, L.Nout, src_map, wgt, meta, d->N, d->n,
-                                                d->i0, d->i0 + d->k, kMetaInts, stream, 1, -1, nullptr, dst_map);
+        j.base0 = Kc; j.base1 = Vc; j.stride_b = kv_sb * 2; j.stride_g = kv_sh * 2; j.G = d->Hkv;
+        j.V = kHeadDim / 8;
+        j.src_map = src_map; j.map_stride = d->N; j.meta = meta; j.meta_stride = kMetaInts;
+        j.Nout = L.Nout; j.merged_row = d->i0 + d->k; j.partial = kv_partial; j.P = L.kvP;
+    }
+    j.B = d->B; j.N = d->N;
+    if (Kc || hidden_out) {
+        const lvlm_status st = launch_inplace_compact(j, stream);
         if (st != LVLM_OK) return st;
     }
     return LVLM_OK;

@@ -640,8 +640,11 @@ lvlm_status launch_nearest_kept(const void* hidden, void* hidden_out, void* Kc, 
                            static_cast<const uint4*>(Vc), kv_sb / 8, kv_sh / 8, d->Hkv, d->N, d->i0, d->k, L.r, kept,
                            drop, order, seg, mass, kvtmp);
         if (st != LVLM_OK) return st;
-        st = launch_inplace_compact(Kc, Vc, kv_sb * 2, kv_sh * 2, d->B, d->Hkv, kHeadDim / 8, L.Nout, src_map, nullptr,
-                                    meta, d->N, d->n, d->i0, 0, kMetaInts, stream);
+        CompactJob cj;
+        cj.base0 = Kc; cj.base1 = Vc; cj.stride_b = kv_sb * 2; cj.stride_g = kv_sh * 2; cj.B = d->B; cj.G = d->Hkv;
+        cj.V = kHeadDim / 8; cj.src_map = src_map; cj.map_stride = d->N; cj.meta = meta; cj.meta_stride = kMetaInts;
+        cj.Nout = L.Nout; cj.N = d->N;
+        st = launch_inplace_compact(cj, stream);
         if (st != LVLM_OK) return st;
         st = launch_kernel(nk_kv_store_kernel, grid, dim3(kNkThreads), 0, stream, 1, static_cast<uint4*>(Kc),
                            static_cast<uint4*>(Vc), kv_sb / 8, kv_sh / 8, d->Hkv, d->i0, d->k, kvtmp);

@@ -10,7 +10,7 @@
 namespace lvlm {
 namespace sm100 {
 
-constexpr uint32_t kSpinLimit = 1u << 24;        // polls of mbarrier.try_wait before giving up
+constexpr uint32_t kSpinLimit = 1u << 21;        // polls of mbarrier.try_wait before giving up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -33,16 +33,18 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
     asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}"
                  ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Returns false if the phase with the given parity did not complete within the poll limit.
+// Returns false if the phase with the given parity did not complete within the poll limit.  A poll that finds
+// the phase incomplete parks the thread (up to about a microsecond; it resumes as soon as the phase completes),
+// so that waiting warps leave the issue slots to the warps that work.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_u32(bar);
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+            : "=r"(done) : "r"(addr), "r"(parity), "r"(1000u) : "memory");
         if (done) return true;
     }
     return false;
@@ -68,6 +70,27 @@ __device__ __forceinline__ void tma_load_3d(void* smem, const CUtensorMap* m, ui
         ::"r"(smem_u32(smem)), "l"(m), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+
+// ---- bulk copies of contiguous bytes (no tensor map) ------------------------------------------
+// Global -> this CTA's shared memory; `bytes` (a multiple of 16) are credited to `bar` when they
+// have landed.  Both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_load(void* smem, const void* gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(smem)), "l"(gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Shared memory -> global, part of the issuing thread's current bulk group.
+__device__ __forceinline__ void bulk_store(void* gmem, const void* smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(gmem), "r"(smem_u32(smem)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// At most N of this thread's bulk groups may still be READING their shared-memory source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// At most N of this thread's bulk groups may still be incomplete.
+template <int N>
+__device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
 
 // ---- tensor memory ---------------------------------------------------------------------------
 // Whole warp.  Writes the base address of `ncols` (power of two >= 32) columns to *dst (smem).
