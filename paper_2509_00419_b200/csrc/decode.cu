@@ -4,32 +4,40 @@
 // the group.
 //
 // One launch, split-K inside thread-block clusters.  The S CTAs of a cluster share one (sequence,
-// KV head): its ceil(len/16) key tiles are cut into S equal runs, so a ragged cache costs what
-// its own length costs.  Inside a CTA every warp streams its tiles through a private ring of
-// shared-memory stages (cp.async, 16-byte chunks XOR-swizzled so that ldmatrix is conflict free),
-// multiplies them with small tensor-core MMAs (the G query heads of the group are the rows of a
-// 16-row tile) and keeps an online softmax per head, so the main loop has no block barrier.  The
-// warps of a CTA are merged in warp order in shared memory; the CTAs of the cluster then read each
-// other's (max, sum, output) through distributed shared memory in rank order, each finishing a
-// slice of the output channels and the acc_score entries of its own keys.  Nothing goes through
-// global scratch except the scaled logits a CTA parks for its own acc_score update.
+// KV head): its key tiles are cut into S equal runs, so a ragged cache costs what its own length
+// costs.  A CTA is one producer warp and four compute warps around a ring of shared-memory stages
+// of 64 keys: the producer fetches the K and V rows of a stage with four TMA tile copies (128-byte
+// swizzle, so that ldmatrix is conflict free; completion counted by an mbarrier), a compute warp
+// takes 16 keys of the stage, multiplies them with small tensor-core MMAs (the G query heads of the
+// group are the rows of a 16-row tile) and keeps an online softmax per head, so the main loop has no
+// block barrier.  With d->cache_stable the first lap of the ring is fetched before the kernel waits
+// for the one ahead of it in the stream.  The warps of a CTA are merged in warp order
+// in shared memory; the CTAs of the cluster then read each other's (max, sum, output) through
+// distributed shared memory in rank order, each finishing a slice of the output channels and the
+// acc_score entries of its own keys, whose scaled logits it has kept in shared memory (in the
+// workspace when a run is too long for that).
 #include <mutex>
 
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace lvlm {
 
-constexpr int kDecThreads = 128;
-constexpr int kDecWarps = 4;
+using namespace sm100;
+
+constexpr int kDecWarps = 4;                         // compute warps
+constexpr int kDecThreads = (kDecWarps + 1) * 32;    // ... and the producer warp
 constexpr int kTileKeys = 16;                        // keys per warp tile
-constexpr int kStagesDec = 3;                        // stages per warp
-constexpr int kTileHalf = kTileKeys * 256;           // bytes of one K (or V) tile
-constexpr int kStageBytes = 2 * kTileHalf;           // K tile then V tile
-constexpr int kRingBytes = kDecWarps * kStagesDec * kStageBytes;
+constexpr int kStageKeys = kDecWarps * kTileKeys;    // keys per stage
+constexpr int kBoxBytes = kStageKeys * 128;          // one TMA box: 64 keys x 64 channels
+constexpr int kStageBytes = 4 * kBoxBytes;           // K low half, K high half, V low half, V high half
+constexpr int kStagesDec = 3;
+constexpr int kRingBytes = kStagesDec * kStageBytes;
 constexpr int kDecAccFloats = 2048;                  // shared floats for merging the warps of a CTA (8 KB)
 constexpr int kDecTargetCtas = 2 * 148;              // CTAs wanted in flight: two per SM of a 148-SM part
 constexpr int kDecMaxCluster = 8;                    // portable cluster size
-constexpr int kDecMinTiles = 4;                      // a CTA's run is not made shorter than this by splitting
+constexpr int kDecMinTiles = 2;                      // a CTA's run is not made shorter than this by splitting
+constexpr int kDecLogitBytes = 12 * 1024;            // scaled logits of a CTA's own keys kept in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct DecodeLayout { int S; size_t off_s, total; };
@@ -87,14 +95,6 @@ __device__ __forceinline__ float dsmem_ld(uint32_t addr) {
     return v;
 }
 
-// 16-byte asynchronous copy; src_bytes = 0 writes zeros instead.
-__device__ __forceinline__ void cp_async16_zfill(uint32_t smem, const void* gmem, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem), "l"(gmem), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];\n"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -118,18 +118,28 @@ struct DecodeArgs {
     const __nv_bfloat16* k_new; const __nv_bfloat16* v_new; float* acc_score; __nv_bfloat16* out;
     int H, Hkv, cap, S;
     int early;               // the cache and len are not written by the kernel ahead: fetch before waiting for it
+    int logit_keys;          // keys of a run whose logits fit in shared memory (0: they go to ws_s)
     int64_t kv_sb, kv_sh;
     float scale_log2;
-    float* ws_s;             // [B*H][cap] scaled logits (log2 domain), only with acc_score
+    float* ws_s;             // [B*H][cap] scaled logits (log2 domain), only with acc_score and a long run
     int32_t* dev_status;
 };
 
+// Offset inside a stage of the 16-byte chunk `ch` (0..15) of key row `r` (0..63): K or V half boxes of 64
+// channels, rows of 128 bytes, chunks XOR-swizzled with the row as the TMA copy wrote them.
+__device__ __forceinline__ uint32_t stage_off(int r, int ch) {
+    return (uint32_t)((ch >> 3) * kBoxBytes + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
+}
+
 // grid.x = heads * S, clusters of S CTAs along x: cluster = (sequence, KV head), rank = run of tiles.
 template <int G>
-__global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const DecodeArgs a) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    float* s_acc = reinterpret_cast<float*>(smem + kRingBytes);         // [slots][G][128]; slot 0 = this CTA's output
-    float* s_wm = s_acc + kDecAccFloats;                                // [4 warps][8 heads] running max
+__global__ void __launch_bounds__(kDecThreads, 2)
+decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
+                      const DecodeArgs a) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    float* s_acc = reinterpret_cast<float*>(smem);                      // [slots][G][128]; slot 0 = this CTA's output (the ring, once it is done)
+    float* s_wm = reinterpret_cast<float*>(smem + kRingBytes);          // [4 warps][8 heads] running max
     float* s_wl = s_wm + kDecWarps * 8;                                 // [4 warps][8 heads] running sum
     float* s_M = s_wl + kDecWarps * 8;                                  // [8] this CTA's max per head
     float* s_L = s_M + 8;                                               // [8] this CTA's sum per head
@@ -137,11 +147,21 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
     float* s_FI = s_FM + 8;                                             // [8] 1 / cluster-wide sum
     float* s_rm = s_FI + 8;                                             // [S][8] max of every CTA of the cluster
     float* s_rl = s_rm + 8 * kDecMaxCluster;                            // [S][8] sum of every CTA
+    uint64_t* s_full = reinterpret_cast<uint64_t*>(s_rl + 8 * kDecMaxCluster);   // [kStagesDec]
+    uint64_t* s_empty = s_full + kStagesDec;                            // [kStagesDec]
+    float* s_logit = reinterpret_cast<float*>(s_empty + kStagesDec + 1);          // [G][logit_keys]
+    __shared__ int s_abort;
 
-    // With a.early the first key/value tiles and the length are fetched while the kernel ahead in the
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < kStagesDec; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kDecWarps); }
+        s_abort = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    // With a.early the first key/value stages and the length are fetched while the kernel ahead in the
     // stream is still finishing; q, k_new, v_new and every write come after the wait in any case.
     if (!a.early) pdl_enter();
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.S, H = a.H, cap = a.cap;
     const int hd = blockIdx.x / S;
     const int rank = (int)cluster_ctarank();
@@ -163,153 +183,180 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
         return;
     }
     const int nt = (lne + kTileKeys - 1) / kTileKeys;
-    const int per = (nt + S - 1) / S;
+    int per = (nt + S - 1) / S;
+    if (per >= kDecWarps) per = (per + kDecWarps - 1) / kDecWarps * kDecWarps;   // whole stages where the run is long enough
     const int t_lo = min(nt, rank * per), t_hi = min(nt, t_lo + per);   // my run of tiles
-
-    if (a.acc_score) {                         // my keys' acc_score entries: needed at the very end, fetched now
-        const float* acc = a.acc_score + (int64_t)hd * cap;
-        const int j_lo = t_lo * kTileKeys, j_hi = min(lne, t_hi * kTileKeys);
-        for (int j = j_lo + tid * 32; j < j_hi; j += kDecThreads * 32) prefetch_l2(acc + j);
-    }
-    const int64_t kv_off = (int64_t)b * a.kv_sb + (int64_t)g * a.kv_sh;
-    __nv_bfloat16* Kseq = a.Kc + kv_off;
-    __nv_bfloat16* Vseq = a.Vc + kv_off;
-    const __nv_bfloat16* kn = app ? a.k_new + (int64_t)hd * kHeadDim : nullptr;
-    const __nv_bfloat16* vn = app ? a.v_new + (int64_t)hd * kHeadDim : nullptr;
-
-    const int row = lane >> 2, qd = lane & 3;
-    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem) + warp * (kStagesDec * kStageBytes);
-    const int my_ntile = (t_hi - t_lo) > warp ? (t_hi - t_lo - warp + kDecWarps - 1) / kDecWarps : 0;
-
-    auto issue = [&](int it) {                 // my it-th tile -> stage it % kStagesDec
-        const uint32_t st = ring + (it % kStagesDec) * kStageBytes;
-        const int j0 = (t_lo + warp + it * kDecWarps) * kTileKeys;
-        // 16 rows x 16 chunks per tensor = 256 chunks, 8 per lane per tensor
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int e = u * 32 + lane;
-            const int r = e >> 4, ch = e & 15;
-            const int j = j0 + r;
-            const bool ok = j < ln;            // rows the cache already holds; an appended row is put in place later
-            const int64_t ro = (int64_t)(ok ? j : 0) * kHeadDim + ch * 8;
-            const uint32_t off = r * 256 + ((ch ^ (r & 7)) << 4);
-            cp_async16_zfill(st + off, Kseq + ro, ok ? 16 : 0);
-            cp_async16_zfill(st + kTileHalf + off, Vseq + ro, ok ? 16 : 0);
-        }
+    const int nstage = (t_hi - t_lo + kDecWarps - 1) / kDecWarps;
+    const uint32_t ring = smem_u32(smem);
+    volatile int* abort_flag = &s_abort;
+    auto wait_on = [&](uint64_t* bar, uint32_t parity) -> bool {
+        if (*abort_flag) return false;
+        if (mbar_wait(bar, parity)) return true;
+        *abort_flag = 1;
+        if (a.dev_status) atomicOr(a.dev_status, LVLM_DEV_TIMEOUT);
+        return false;
     };
-#pragma unroll
-    for (int it = 0; it < kStagesDec - 1; ++it) {
-        if (it < my_ntile) issue(it);
-        cp_async_commit();
-    }
 
-    if (a.early) pdl_enter();
-    // query fragments: heads of the group are rows 0..G-1 of a 16-row A tile
-    uint32_t qa[8][2];
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-        qa[ks][0] = qa[ks][1] = 0u;
-        if (row < G) {
-            const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q + (int64_t)(b * H + h0 + row) * kHeadDim);
-            qa[ks][0] = __ldg(qp + ks * 8 + qd);
-            qa[ks][1] = __ldg(qp + ks * 8 + 4 + qd);
-        }
-    }
     float o[16][2];                            // head `row`, columns nt*8 + qd*2 + {0,1}
 #pragma unroll
     for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = 0.f;
     float m_run = -INFINITY, l_run = 0.f;      // of head `row`; l_run is this lane's share of the sum
+    const int row = lane >> 2, qd = lane & 3;
 
-    for (int it = 0; it < my_ntile; ++it) {
-        cp_async_wait<kStagesDec - 2>();
-        __syncwarp();
-        const uint32_t st = ring + (it % kStagesDec) * kStageBytes;
-        const int j0 = (t_lo + warp + it * kDecWarps) * kTileKeys;
-        if (app && ln >= j0 && ln < j0 + kTileKeys) {
-            // the appended row: into its place of the tile (zero-filled by the copy) and into the cache
-            const int rr = ln - j0, ch = lane & 15;
-            const uint4 x = *reinterpret_cast<const uint4*>((lane < 16 ? kn : vn) + ch * 8);
-            const uint32_t off = (lane < 16 ? 0 : kTileHalf) + rr * 256 + ((ch ^ (rr & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st + off), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
-            *reinterpret_cast<uint4*>((lane < 16 ? Kseq : Vseq) + (int64_t)ln * kHeadDim + ch * 8) = x;
+    if (warp == kDecWarps) {
+        // ---- producer: four tile copies per stage ---------------------------------------------------------
+        auto issue = [&](int s) {
+            unsigned char* st = smem + (s % kStagesDec) * kStageBytes;
+            const int j0 = (t_lo + s * kDecWarps) * kTileKeys;
+            mbar_arrive_expect_tx(&s_full[s % kStagesDec], kStageBytes);
+            tma_load_4d(st, &kmap, &s_full[s % kStagesDec], 0, j0, g, b);
+            tma_load_4d(st + kBoxBytes, &kmap, &s_full[s % kStagesDec], 64, j0, g, b);
+            tma_load_4d(st + 2 * kBoxBytes, &vmap, &s_full[s % kStagesDec], 0, j0, g, b);
+            tma_load_4d(st + 3 * kBoxBytes, &vmap, &s_full[s % kStagesDec], 64, j0, g, b);
+        };
+        if (lane == 0) {
+            prefetch_tmap(&kmap);
+            prefetch_tmap(&vmap);
+            for (int s = 0; s < kStagesDec && s < nstage; ++s) issue(s);
+        }
+        if (a.early) pdl_enter();
+        if (lane == 0) {
+            for (int s = kStagesDec; s < nstage; ++s) {
+                if (!wait_on(&s_empty[s % kStagesDec], (uint32_t)(s / kStagesDec - 1) & 1u)) break;
+                issue(s);
+            }
+        }
+    } else {
+        if (a.acc_score) {                     // my keys' acc_score entries: needed at the very end, fetched now
+            const float* acc = a.acc_score + (int64_t)hd * cap;
+            const int j_lo = t_lo * kTileKeys, j_hi = min(lne, t_hi * kTileKeys);
+            for (int j = j_lo + tid * 32; j < j_hi; j += kDecWarps * 32 * 32) prefetch_l2(acc + j);
+        }
+        if (a.early) pdl_enter();
+        const int64_t kv_off = (int64_t)b * a.kv_sb + (int64_t)g * a.kv_sh;
+        __nv_bfloat16* Kseq = a.Kc + kv_off;
+        __nv_bfloat16* Vseq = a.Vc + kv_off;
+        const __nv_bfloat16* kn = app ? a.k_new + (int64_t)hd * kHeadDim : nullptr;
+        const __nv_bfloat16* vn = app ? a.v_new + (int64_t)hd * kHeadDim : nullptr;
+        // query fragments: heads of the group are rows 0..G-1 of a 16-row A tile
+        uint32_t qa[8][2];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qa[ks][0] = qa[ks][1] = 0u;
+            if (row < G) {
+                const uint32_t* qp = reinterpret_cast<const uint32_t*>(a.q + (int64_t)(b * H + h0 + row) * kHeadDim);
+                qa[ks][0] = __ldg(qp + ks * 8 + qd);
+                qa[ks][1] = __ldg(qp + ks * 8 + 4 + qd);
+            }
+        }
+        for (int s = 0; s < nstage; ++s) {
+            const bool ok = wait_on(&s_full[s % kStagesDec], (uint32_t)(s / kStagesDec) & 1u);
+            const int t = t_lo + s * kDecWarps + warp;
+            if (ok && t < t_hi) {
+                const uint32_t st = ring + (s % kStagesDec) * kStageBytes;      // K boxes; the V boxes follow
+                const int r0 = warp * kTileKeys;                               // my rows of the stage
+                const int j0 = t * kTileKeys;
+                if (app && ln >= j0 && ln < j0 + kTileKeys) {
+                    // the appended row: into its place of the tile and into the cache
+                    const int rr = r0 + ln - j0, ch = lane & 15;
+                    const uint4 x = *reinterpret_cast<const uint4*>((lane < 16 ? kn : vn) + ch * 8);
+                    const uint32_t off = (lane < 16 ? 0 : 2 * kBoxBytes) + stage_off(rr, ch);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st + off), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
+                    *reinterpret_cast<uint4*>((lane < 16 ? Kseq : Vseq) + (int64_t)ln * kHeadDim + ch * 8) = x;
+                }
+                if (j0 + kTileKeys > lne) {
+                    // V rows past the last key hold whatever the cache holds: zero them, their weight is zero
+                    for (int e = lane; e < (j0 + kTileKeys - lne) * 16; e += 32) {
+                        const int rr = r0 + (lne - j0) + (e >> 4), ch = e & 15;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(st + 2 * kBoxBytes + stage_off(rr, ch)), "r"(0u) : "memory");
+                    }
+                }
+                __syncwarp();
+                // ---- S = Q K^T for 16 keys -------------------------------------------------------------------
+                float sc[2][4];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f;
+                {
+                    const int mi = lane >> 3, r8 = lane & 7;
+                    const int key = r0 + (mi >> 1) * 8 + r8;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int chunkc = 2 * ks + (mi & 1);
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4(st + stage_off(key, chunkc), b0, b1, b2, b3);
+                        mma_16816(sc[0], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+                        mma_16816(sc[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+                    }
+                }
+                // ---- online softmax of head `row` over the tile's keys -------------------------------------------
+                float tmax = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc) {
+                        const int j = j0 + i * 8 + qd * 2 + cc;
+                        float v = sc[i][cc] * a.scale_log2;
+                        if (j >= lne) v = -INFINITY;
+                        sc[i][cc] = v;
+                        tmax = fmaxf(tmax, v);
+                        if (a.acc_score && row < G && j < lne) {
+                            if (a.logit_keys) s_logit[row * a.logit_keys + (j - t_lo * kTileKeys)] = v;
+                            else a.ws_s[(int64_t)(b * H + h0 + row) * cap + j] = v;
+                        }
+                    }
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 1));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 2));
+                const float m_new = fmaxf(m_run, tmax);          // finite: every tile has a valid key
+                const float corr = exp2f(m_run - m_new);
+                m_run = m_new;
+                float p[2][2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc) p[i][cc] = exp2f(sc[i][cc] - m_new);
+                l_run = l_run * corr + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
+                // ---- O += P V -----------------------------------------------------------------------------------
+                // P is split into a bf16 head and a bf16 remainder so that the product keeps ~16 bits
+                const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]), pa2 = pack_bf16(p[1][0], p[1][1]);
+                const uint32_t pr0 = pack_bf16(p[0][0] - bf16_lo(pa0), p[0][1] - bf16_hi(pa0));
+                const uint32_t pr2 = pack_bf16(p[1][0] - bf16_lo(pa2), p[1][1] - bf16_hi(pa2));
+                {
+                    const int mi = lane >> 3, r8 = lane & 7;
+                    const int key = r0 + (mi & 1) * 8 + r8;
+#pragma unroll
+                    for (int dp = 0; dp < 8; ++dp) {
+                        const int chunkc = 2 * dp + (mi >> 1);
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4_trans(st + 2 * kBoxBytes + stage_off(key, chunkc), b0, b1, b2, b3);
+                        // rows 8..15 of the MMA tile are padding: their accumulators are thrown away
+                        float d0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
+                        float d1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
+                        mma_16816(d0, pa0, 0u, pa2, 0u, b0, b1);
+                        mma_16816(d1, pa0, 0u, pa2, 0u, b2, b3);
+                        mma_16816(d0, pr0, 0u, pr2, 0u, b0, b1);
+                        mma_16816(d1, pr0, 0u, pr2, 0u, b2, b3);
+                        o[2 * dp][0] = d0[0]; o[2 * dp][1] = d0[1];
+                        o[2 * dp + 1][0] = d1[0]; o[2 * dp + 1][1] = d1[1];
+                    }
+                }
+            }
             __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[s % kStagesDec]);
         }
-        // ---- S = Q K^T for 16 keys -------------------------------------------------------------------
-        float s[2][4];
-#pragma unroll
-        for (int i = 0; i < 2; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
-        {
-            const int mi = lane >> 3, r8 = lane & 7;
-            const int key = (mi >> 1) * 8 + r8;
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const int chunkc = 2 * ks + (mi & 1);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4(st + key * 256 + ((chunkc ^ (key & 7)) << 4), b0, b1, b2, b3);
-                mma_16816(s[0], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
-                mma_16816(s[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
-            }
-        }
-        // ---- online softmax of head `row` over the tile's keys -------------------------------------------
-        float tmax = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < 2; ++i)
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                const int j = j0 + i * 8 + qd * 2 + cc;
-                float v = s[i][cc] * a.scale_log2;
-                if (j >= lne) v = -INFINITY;
-                s[i][cc] = v;
-                tmax = fmaxf(tmax, v);
-                if (a.ws_s && row < G && j < lne) a.ws_s[(int64_t)(b * H + h0 + row) * cap + j] = v;
-            }
-        tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 1));
-        tmax = fmaxf(tmax, __shfl_xor_sync(0xFFFFFFFFu, tmax, 2));
-        const float m_new = fmaxf(m_run, tmax);          // finite: every tile has a valid key
-        const float corr = exp2f(m_run - m_new);
-        m_run = m_new;
-        float p[2][2];
-#pragma unroll
-        for (int i = 0; i < 2; ++i)
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) p[i][cc] = exp2f(s[i][cc] - m_new);
-        l_run = l_run * corr + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
-        // ---- O += P V -----------------------------------------------------------------------------------
-        // P is split into a bf16 head and a bf16 remainder so that the product keeps ~16 bits
-        const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]), pa2 = pack_bf16(p[1][0], p[1][1]);
-        const uint32_t pr0 = pack_bf16(p[0][0] - bf16_lo(pa0), p[0][1] - bf16_hi(pa0));
-        const uint32_t pr2 = pack_bf16(p[1][0] - bf16_lo(pa2), p[1][1] - bf16_hi(pa2));
-        {
-            const int mi = lane >> 3, r8 = lane & 7;
-            const int key = (mi & 1) * 8 + r8;
-#pragma unroll
-            for (int dp = 0; dp < 8; ++dp) {
-                const int chunkc = 2 * dp + (mi >> 1);
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4_trans(st + kTileHalf + key * 256 + ((chunkc ^ (key & 7)) << 4), b0, b1, b2, b3);
-                // rows 8..15 of the MMA tile are padding: their accumulators are thrown away
-                float d0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
-                float d1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
-                mma_16816(d0, pa0, 0u, pa2, 0u, b0, b1);
-                mma_16816(d1, pa0, 0u, pa2, 0u, b2, b3);
-                mma_16816(d0, pr0, 0u, pr2, 0u, b0, b1);
-                mma_16816(d1, pr0, 0u, pr2, 0u, b2, b3);
-                o[2 * dp][0] = d0[0]; o[2 * dp][1] = d0[1];
-                o[2 * dp + 1][0] = d1[0]; o[2 * dp + 1][1] = d1[1];
-            }
-        }
-        __syncwarp();
-        if (it + kStagesDec - 1 < my_ntile) issue(it + kStagesDec - 1);
-        cp_async_commit();
     }
-    cp_async_wait<0>();
+    // every copy issued has landed: the compute warps have waited for each stage; the ring is free
+    __syncthreads();
+    if (s_abort) {                             // a wait gave up: copies may still be in flight, let them land
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
 
     // ---- merge the four warps in warp order ------------------------------------------------------------
     l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
     l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-    if (row < G && qd == 0) { s_wm[warp * 8 + row] = m_run; s_wl[warp * 8 + row] = l_run; }
+    if (warp < kDecWarps && row < G && qd == 0) { s_wm[warp * 8 + row] = m_run; s_wl[warp * 8 + row] = l_run; }
     __syncthreads();
     {
         // kSlots warps write side by side, the others add to them in warp order; the slots are added
@@ -336,7 +383,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
             __syncthreads();
         }
 #pragma unroll
-        for (int hh = 0; hh < G; ++hh) {                  // thread = channel
+        for (int hh = 0; hh < G && tid < kHeadDim; ++hh) {  // thread = channel
             float v = s_acc[hh * kHeadDim + tid];
 #pragma unroll
             for (int sl = 1; sl < kSlots; ++sl) v += s_acc[sl * (G * kHeadDim) + hh * kHeadDim + tid];
@@ -430,7 +477,8 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_cluster_kernel(const De
                 if (j < j_hi) {
 #pragma unroll
                     for (int hh = 0; hh < G; ++hh)
-                        lg[u][hh] = __ldcg(a.ws_s + (int64_t)(b * H + h0 + hh) * cap + j);
+                        lg[u][hh] = a.logit_keys ? s_logit[hh * a.logit_keys + (j - j_lo)]
+                                                 : __ldcg(a.ws_s + (int64_t)(b * H + h0 + hh) * cap + j);
                     if (!(app && j == ln)) old[u] = acc[j];                  // a new entry starts at zero
                 }
             }
@@ -455,10 +503,24 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
                                  const void* v_new, float* acc_score, const lvlm_dims* d, float scale,
                                  void* out, char* wsb, const DecodeLayout& L, int64_t kv_sb,
                                  int64_t kv_sh, int32_t* dev_status, cudaStream_t stream) {
-    const size_t smem = (size_t)kRingBytes + (size_t)(kDecAccFloats + 2 * kDecWarps * 8 + 4 * 8 +
-                                                      3 * 8 * kDecMaxCluster) * 4;
+    // scaled logits of a CTA's own keys stay in shared memory when the longest run fits the budget
+    const int nt_max = (d->cap + kTileKeys - 1) / kTileKeys;
+    int per = (nt_max + L.S - 1) / L.S;
+    if (per >= kDecWarps) per = (per + kDecWarps - 1) / kDecWarps * kDecWarps;
+    const int run_keys = per * kTileKeys;
+    const int logit_keys = acc_score && (size_t)G * run_keys * 4 <= (size_t)kDecLogitBytes ? run_keys : 0;
+    const size_t smem = 1024 + (size_t)kRingBytes + (size_t)(2 * kDecWarps * 8 + 4 * 8 + 2 * 8 * kDecMaxCluster) * 4 +
+                        (size_t)(2 * kStagesDec + 1) * 8 + (size_t)G * logit_keys * 4;
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(decode_cluster_kernel<G>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+    CUtensorMap kmap, vmap;
+    {
+        const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)d->cap, (uint64_t)d->Hkv, (uint64_t)d->B};
+        const uint64_t strides[3] = {(uint64_t)kHeadDim * 2, (uint64_t)kv_sh * 2, (uint64_t)kv_sb * 2};
+        const uint32_t box[4] = {64, (uint32_t)kStageKeys, 1, 1};
+        if (!make_tmap_bf16(&kmap, Kc, 4, dims, strides, box) || !make_tmap_bf16(&vmap, Vc, 4, dims, strides, box))
+            return LVLM_ERR_CUDA;
+    }
     const int64_t ctas = (int64_t)d->B * d->Hkv * L.S;
     if (ctas > 0x7FFFFFFFll) return LVLM_ERR_UNSUPPORTED;
     DecodeArgs a;
@@ -474,9 +536,10 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
     a.early = d->cache_stable != 0 && pdl_enabled();
     a.kv_sb = kv_sb; a.kv_sh = kv_sh; a.scale_log2 = scale * kLog2e;
     a.ws_s = acc_score ? reinterpret_cast<float*>(wsb + L.off_s) : nullptr;
+    a.logit_keys = logit_keys;
     a.dev_status = dev_status;
 
-    return launch_kernel(decode_cluster_kernel<G>, dim3((unsigned)ctas), dim3(kDecThreads), smem, stream, L.S, a);
+    return launch_kernel(decode_cluster_kernel<G>, dim3((unsigned)ctas), dim3(kDecThreads), smem, stream, L.S, kmap, vmap, a);
 }
 
 }  // namespace lvlm

@@ -34,7 +34,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
                  ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 // Returns false if the phase with the given parity did not complete within the poll limit.  A poll that finds
-// the phase incomplete parks the thread (up to about a microsecond; it resumes as soon as the phase completes),
+// the phase incomplete parks the thread for a moment (it resumes as soon as the phase completes),
 // so that waiting warps leave the issue slots to the warps that work.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_u32(bar);
@@ -44,7 +44,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
             "{\n\t.reg .pred p;\n\t"
             "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity), "r"(1000u) : "memory");
+            : "=r"(done) : "r"(addr), "r"(parity), "r"(64u) : "memory");
         if (done) return true;
     }
     return false;
