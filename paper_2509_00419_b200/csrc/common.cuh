@@ -10,7 +10,7 @@
 namespace lvlm {
 
 constexpr int kHeadDim = 128;
-constexpr int kMaxSortN = 16384;      // kv_compress: one CTA sorts at most this many 64-bit keys in shared memory
+constexpr int kMaxSortN = 16384;      // kv_compress: one CTA (1024 threads, 16 entries each) holds at most this many keys
 constexpr int kMaxGroup = 8;          // query heads per KV head supported by decode attention
 // Opt-in limit of dynamic shared memory asked for every kernel that may exceed 48 KB.  The
 // attribute is a property of the function, not of a launch, so it is always set to this one

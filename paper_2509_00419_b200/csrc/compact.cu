@@ -31,6 +31,7 @@ struct InplaceArgs {
     int G, T, V, Vsub, S, Nout, meta_stride, maps_per_g, Rmax, CG, RL, merged_row, P;
     const int32_t* src_map; const int32_t* meta; const int32_t* nout; const float* partial;
     char* fin_base; int64_t fin_stride_b; int fin_row, fin_V, fin_P, fin_y; const float* fin_partial;
+    uint32_t* side_dst[2]; const uint32_t* side_src[2];
 };
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
@@ -107,6 +108,12 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
     const int CG = a.CG, RL = a.RL;
     const int cg = threadIdx.x % CG, rl = threadIdx.x / CG;
 
+    // the small per-entry arrays the kernel before compacted out of place: copied back by the CTA of tensor `which`
+    if (col == 0 && rank == 0 && which < 2 && a.side_dst[which]) {
+        uint32_t* sd = a.side_dst[which] + (int64_t)m * a.map_stride;
+        const uint32_t* ss = a.side_src[which] + (int64_t)m * a.map_stride;
+        for (int o = o_start + threadIdx.x; o < Nout; o += kCompactThreads) sd[o] = ss[o];
+    }
     // positions per CTA per super-tile: everything that is left, shared out evenly, capped by the buffer
     int R = (max(Nout - o_start, 1) + S - 1) / S;
     R = (R + RL - 1) / RL * RL;
@@ -214,6 +221,11 @@ lvlm_status launch_inplace_compact(const CompactJob& j, cudaStream_t stream) {
     a.src_map = j.src_map; a.meta = j.meta; a.nout = j.nout;
     a.merged_row = j.merged_row; a.partial = j.partial; a.P = j.P;
     if (fin) a.fin_y = j.G * a.T;
+    for (int i = 0; i < 2; ++i) {
+        a.side_dst[i] = static_cast<uint32_t*>(j.side_dst[i]);
+        a.side_src[i] = static_cast<const uint32_t*>(j.side_src[i]);
+    }
+    if (a.side_dst[1] && !j.base1) return LVLM_ERR_INVALID_ARG;   // the second array rides with the second tensor
 
     // enough CTAs to fill the GPU: first a cluster per sequence, then column groups of wide rows
     const int64_t nseq = (int64_t)j.B * j.G * a.T;

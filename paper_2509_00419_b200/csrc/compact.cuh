@@ -27,6 +27,10 @@ struct CompactJob {
     int merged_row = -1;
     const float* partial = nullptr;
     int P = 0;
+    // Optionally up to two arrays of 4-byte words per sequence map (maps_per_g != 1), rows map_stride words apart:
+    // words [meta, nout) of side_src[i] are copied to side_dst[i] (compacted out of place by the kernel before).
+    void* side_dst[2] = {nullptr, nullptr};
+    const void* side_src[2] = {nullptr, nullptr};
     // Optionally, in the same launch: row `fin_row` of every sequence of another tensor (rows of fin_V 16-byte
     // vectors, sequences fin_stride_b bytes apart) receives the sum of the fin_P partial rows
     // fin_partial[(b*fin_P + p)*fin_V*8 ...].  base0 may be NULL then: nothing is compacted.

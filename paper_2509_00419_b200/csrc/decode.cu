@@ -153,6 +153,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 32) { prefetch_tmap(&kmap); prefetch_tmap(&vmap); }     // the descriptors start their way first
     if (tid == 0) {
         for (int s = 0; s < kStagesDec; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kDecWarps); }
         s_abort = 0;
@@ -215,8 +216,6 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             tma_load_4d(st + 3 * kBoxBytes, &vmap, &s_full[s % kStagesDec], 64, j0, g, b);
         };
         if (lane == 0) {
-            prefetch_tmap(&kmap);
-            prefetch_tmap(&vmap);
             for (int s = 0; s < kStagesDec && s < nstage; ++s) issue(s);
         }
         if (a.early) pdl_enter();

@@ -1,16 +1,15 @@
 // lvlm_kv_compress: per (sequence, KV head) eviction of low-score cache entries
 // (Section 3.2.2, paragraph 2: sort the scores in descending order, keep the entries whose
 // accumulated score reaches the threshold beta, discard the other image entries; Appendix A.2:
-// beta = 0.995).  A plan kernel ranks the evictable entries, finds the count, builds the
-// survivor map and compacts the small per-entry arrays; the shared in-place compaction kernel
+// beta = 0.995).  A plan kernel finds the entry at which the threshold (and the budget) is met,
+// builds the survivor map and compacts the small per-entry arrays; the shared in-place compaction kernel
 // then moves the K and V rows.
 #include "common.cuh"
 #include "compact.cuh"
-#include "sort.cuh"
 
 namespace lvlm {
 
-struct KvLayout { size_t off_src, off_meta, off_nout, total; };
+struct KvLayout { size_t off_src, off_meta, off_nout, off_acc, off_pos, total; };
 
 static bool kv_layout(const lvlm_dims* d, KvLayout* L) {
     if (!d || d->B <= 0 || d->Hkv <= 0 || d->cap <= 0 || d->recent < 0) return false;
@@ -19,6 +18,8 @@ static bool kv_layout(const lvlm_dims* d, KvLayout* L) {
     L->off_src = off;  off = align_up(off + heads * d->cap * 4, 256);
     L->off_meta = off; off = align_up(off + heads * 4, 256);
     L->off_nout = off; off = align_up(off + heads * 4, 256);
+    L->off_acc = off;  off = align_up(off + heads * d->cap * 4, 256);     // compacted acc_score and pos, copied back
+    L->off_pos = off;  off = align_up(off + heads * d->cap * 4, 256);     // by the kernel that moves the rows
     L->total = off;
     return true;
 }
@@ -26,35 +27,6 @@ static bool kv_layout(const lvlm_dims* d, KvLayout* L) {
 size_t kv_compress_workspace(const lvlm_dims* d) {
     KvLayout L;
     return kv_layout(d, &L) ? L.total : 0;
-}
-
-// Exclusive prefix sum of one 64-bit integer per thread (same contract as block_exclusive_scan).
-__device__ __forceinline__ long long block_exclusive_scan_ll(long long v, long long* scratch,
-                                                             long long* total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-    long long incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        long long t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    __syncthreads();
-    if (lane == 31) scratch[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        long long w = lane < nwarp ? scratch[lane] : 0;
-        long long wi = w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            long long t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
-            if (lane >= o) wi += t;
-        }
-        scratch[lane] = wi - w;
-        if (lane == 31) scratch[32] = wi;
-    }
-    __syncthreads();
-    *total = scratch[32];
-    return scratch[warp] + incl - v;
 }
 
 // Score in integer units of 2^-24 (negative and non-finite scores count as zero).
@@ -80,84 +52,41 @@ __device__ __forceinline__ unsigned long long ceil_muldiv(unsigned long long a, 
     return q + (rem != 0);
 }
 
-constexpr int kPlanBins = 1024;
-constexpr int kPlanBinFrom = 512;          // evictable sets at least this large are ordered by binned counting
-constexpr int kPlanBinMaxCap = 8192;       // ... when the second key array fits in shared memory
-
-// Ascending order of m distinct 64-bit keys (m <= blockDim.x * 16) without a sorting network: the keys
-// are put into 1024 bins by their high word (linear between the extremes), the place of a key is the
-// number of keys in lower bins plus the number of smaller keys in its own bin.  On return `sorted` holds
-// the keys in order.  srank: m ints, bins: 2 * kPlanBins + 1 ints of shared memory.
-__device__ __forceinline__ void block_order_by_bins(const uint64_t* keys, uint64_t* sorted, int m, int* srank,
-                                                    int* bins, int* scan_scratch) {
-    __shared__ uint32_t s_min[32], s_max[32];
-    int* start = bins;                       // [kPlanBins + 1]
-    int* cursor = bins + kPlanBins + 1;      // [kPlanBins]
-    const int tid = threadIdx.x;
-    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
-    for (int i = tid; i < m; i += blockDim.x) {
-        const uint32_t h = (uint32_t)(keys[i] >> 32);
-        lo = min(lo, h); hi = max(hi, h);
-    }
+// Sums over the block of a count and a 64-bit mass (one barrier: the scratch rows alternate with `turn`).
+struct PlanScratch { int c[2][32]; unsigned long long m[2][32]; };
+__device__ __forceinline__ void block_sum2(int* c, unsigned long long* ms, PlanScratch* sc, int turn) {
+    int cc = *c;
+    unsigned long long mm = *ms;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        lo = min(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
-        hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+        cc += __shfl_xor_sync(0xFFFFFFFFu, cc, o);
+        mm += __shfl_xor_sync(0xFFFFFFFFu, mm, o);
     }
-    if ((tid & 31) == 0) { s_min[tid >> 5] = lo; s_max[tid >> 5] = hi; }
-    for (int i = tid; i <= kPlanBins; i += blockDim.x) start[i] = 0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    if (lane == 0) { sc->c[turn][warp] = cc; sc->m[turn][warp] = mm; }
     __syncthreads();
-    for (int wv = 0; wv < (int)(blockDim.x >> 5); ++wv) { lo = min(lo, s_min[wv]); hi = max(hi, s_max[wv]); }
-    const uint64_t span = (uint64_t)(hi - lo) + 1;
-    auto bin_of = [&](uint32_t h) { return (int)(((uint64_t)(h - lo) * kPlanBins) / span); };
-    for (int i = tid; i < m; i += blockDim.x) atomicAdd(&start[bin_of((uint32_t)(keys[i] >> 32))], 1);
-    __syncthreads();
-    {   // exclusive scan of the bin counts: the first 256 threads take four bins each
-        int c4[4] = {0, 0, 0, 0}, sum = 0;
-        if (tid < kPlanBins / 4) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { c4[u] = start[tid * 4 + u]; sum += c4[u]; }
-        }
-        int total;
-        int run = block_exclusive_scan(sum, scan_scratch, &total);
-        if (tid < kPlanBins / 4) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { start[tid * 4 + u] = run; cursor[tid * 4 + u] = run; run += c4[u]; }
-        }
-        if (tid == 0) start[kPlanBins] = total;
-    }
-    __syncthreads();
-    for (int i = tid; i < m; i += blockDim.x) {
-        const uint64_t key = keys[i];
-        sorted[atomicAdd(&cursor[bin_of((uint32_t)(key >> 32))], 1)] = key;       // bin by bin, any order inside
-    }
-    __syncthreads();
-    for (int i = tid; i < m; i += blockDim.x) {
-        const uint64_t key = keys[i];
-        const int bj = bin_of((uint32_t)(key >> 32));
-        int r = start[bj];
-        for (int p = start[bj]; p < start[bj + 1]; ++p) r += sorted[p] < key;
-        srank[i] = r;
-    }
-    __syncthreads();
-    for (int i = tid; i < m; i += blockDim.x) sorted[srank[i]] = keys[i];
-    __syncthreads();
+    cc = 0; mm = 0;
+    for (int wv = 0; wv < nwarp; ++wv) { cc += sc->c[turn][wv]; mm += sc->m[turn][wv]; }
+    *c = cc; *ms = mm;
 }
 
+// One CTA per (sequence, KV head).  A thread holds KPT consecutive evictable entries as 64-bit keys (order-
+// preserving image of the score above the index: ascending key = descending score, lower index first).  Nothing
+// is sorted: the entry at which the accumulated score reaches the threshold, and the entry that closes the budget,
+// are found by building the key bit by bit from the top - "do the entries up to this key reach the target?" is one
+// sum over the block - and only over the bits in which the keys differ at all.  All sums are integers, so the
+// result does not depend on the order of summation.
+template <int KPT>
 __global__ void __launch_bounds__(1024)
 kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __restrict__ e_lo,
-               const int32_t* __restrict__ e_hi, int Hkv, int cap, int recent, int P_max, int binned,
+               const int32_t* __restrict__ e_hi, int Hkv, int cap, int recent,
                unsigned long long beta_ppm, int budget, int32_t* __restrict__ src_map,
-               int32_t* __restrict__ meta, int32_t* __restrict__ nout, int32_t* dev_status) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* keys = reinterpret_cast<uint64_t*>(smem_raw);
-    int32_t* flag = reinterpret_cast<int32_t*>(keys + P_max);      // [cap]
-    uint64_t* keys2 = reinterpret_cast<uint64_t*>(flag + ((cap + 1) & ~1));            // [P_max], binned only
-    int32_t* bins = reinterpret_cast<int32_t*>(keys2 + P_max);                         // [2 * kPlanBins + 1]
+               int32_t* __restrict__ meta, int32_t* __restrict__ nout, float* __restrict__ acc_new,
+               int32_t* __restrict__ pos_new, int32_t* dev_status) {
+    __shared__ PlanScratch sc;
+    __shared__ unsigned long long s_and[32], s_or[32];
     __shared__ int scan_scratch[33];
-    __shared__ long long scan_ll[33];
-    __shared__ unsigned long long s_thr;
-    __shared__ int s_below, s_first_drop;
+    __shared__ int s_first_drop;
 
     pdl_enter();
     const int g = blockIdx.x, b = blockIdx.y;
@@ -178,74 +107,130 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
     lo = min(max(lo, 0), ln);
     hi = max(hi, lo);
     const int m = hi - lo;
-    int P = 2;
-    while (P < m) P <<= 1;
+    if (threadIdx.x == 0) s_first_drop = m;
+    // compacted acc_score and pos go beside the map; the kernel that moves the K and V rows copies them back
+    float* an = acc_new + (int64_t)m_idx * cap;
+    const int32_t* ps = pos ? pos + (int64_t)m_idx * cap : nullptr;
+    int32_t* pn = pos_new + (int64_t)m_idx * cap;
 
+    // ---- my keys -------------------------------------------------------------------------------------
+    const int j0 = threadIdx.x * KPT;
+    uint64_t key[KPT];
     bool nonfinite = false;
-    if (threadIdx.x == 0) { s_below = 0; s_first_drop = m; }
-    for (int j = threadIdx.x; j < P; j += blockDim.x) {
-        uint64_t key = ~0ull;
-        if (j < m) key = ((uint64_t)desc_key(acc[lo + j], &nonfinite) << 32) | (uint32_t)j;
-        keys[j] = key;
+    uint64_t k_and = ~0ull, k_or = 0ull;
+    unsigned long long total = 0;
+    int turn = 0;
+#pragma unroll
+    for (int u = 0; u < KPT; ++u) {
+        key[u] = ~0ull;                                  // past the end: above every real key
+        if (j0 + u < m) {
+            const float sv = acc[lo + j0 + u];
+            key[u] = ((uint64_t)desc_key(sv, &nonfinite) << 32) | (uint32_t)(j0 + u);
+            k_and &= key[u]; k_or |= key[u];
+            total += (unsigned long long)score_units(sv);
+        }
     }
     if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
-    __syncthreads();
-    if (binned && m >= kPlanBinFrom) {
-        block_order_by_bins(keys, keys2, m, flag, bins, scan_scratch);
-        keys = keys2;
-    } else {
-        block_bitonic_sort(keys, P);
-    }
-
-    // ---- how many entries of E reach the threshold ---------------------------------------
-    int k_beta = m;
-    if (beta_ppm < 1000000ull && m > 0) {
-        const int per = (m + blockDim.x - 1) / blockDim.x;
-        const int p0 = min(m, (int)threadIdx.x * per), p1 = min(m, p0 + per);
-        long long part = 0;
-        for (int p = p0; p < p1; ++p) part += score_units(acc[lo + (int)(uint32_t)keys[p]]);
-        long long total;
-        long long cum = block_exclusive_scan_ll(part, scan_ll, &total);
-        if (threadIdx.x == 0) s_thr = ceil_muldiv(beta_ppm, (unsigned long long)total, 1000000ull);
-        __syncthreads();
-        const unsigned long long thr = s_thr;
-        int below = 0;                                   // prefixes whose sum is still short
-        for (int p = p0; p < p1; ++p) {
-            cum += score_units(acc[lo + (int)(uint32_t)keys[p]]);
-            if ((unsigned long long)cum < thr) ++below;
+    // units of a key's score, recomputed from the key when a sum needs them
+    auto units_of = [](uint64_t k) -> unsigned long long {
+        const uint32_t dk = (uint32_t)(k >> 32);
+        if (dk == 0xFFFFFFFFu) return 0ull;             // NaN (or no entry)
+        const uint32_t asc = ~dk;
+        const uint32_t bits = (asc & 0x80000000u) ? (asc & 0x7FFFFFFFu) : ~asc;
+        return (unsigned long long)score_units(__uint_as_float(bits));
+    };
+    {   // bits in which the keys differ, and the total score
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            k_and &= __shfl_xor_sync(0xFFFFFFFFu, k_and, o);
+            k_or |= __shfl_xor_sync(0xFFFFFFFFu, k_or, o);
         }
-        below = warp_sum(below);
-        if ((threadIdx.x & 31) == 0 && below) atomicAdd(&s_below, below);
-        __syncthreads();
-        k_beta = min(m, s_below + 1);
+        if ((threadIdx.x & 31) == 0) { s_and[threadIdx.x >> 5] = k_and; s_or[threadIdx.x >> 5] = k_or; }
+        int dummy = 0;
+        block_sum2(&dummy, &total, &sc, turn); turn ^= 1;            // (its barrier also publishes s_and / s_or)
+        k_and = ~0ull; k_or = 0ull;
+        for (int wv = 0; wv < (int)(blockDim.x >> 5); ++wv) { k_and &= s_and[wv]; k_or |= s_or[wv]; }
+    }
+    const uint64_t diff = m > 0 ? (k_and ^ k_or) : 0ull;
+    // Smallest key T such that the entries with key <= T hold at least `target` (their count, or their score when
+    // by_mass).  The caller guarantees that all entries together reach the target.
+    auto search = [&](unsigned long long target, bool by_mass) -> uint64_t {
+        uint64_t ans = k_and;
+        uint64_t todo = diff;
+        while (todo) {
+            const int bit = 63 - __clzll((long long)todo);
+            todo &= ~(1ull << bit);
+            const uint64_t cand = (ans & ~(1ull << bit)) | ((1ull << bit) - 1ull);
+            int cnt = 0;
+            unsigned long long ms = 0;
+#pragma unroll
+            for (int u = 0; u < KPT; ++u) {
+                if (key[u] <= cand) { ++cnt; if (by_mass) ms += units_of(key[u]); }
+            }
+            block_sum2(&cnt, &ms, &sc, turn); turn ^= 1;
+            const unsigned long long have = by_mass ? ms : (unsigned long long)cnt;
+            if (have >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
+        }
+        return ans;
+    };
+    auto count_upto = [&](uint64_t T) -> int {
+        int cnt = 0;
+        unsigned long long ms = 0;
+#pragma unroll
+        for (int u = 0; u < KPT; ++u) cnt += key[u] <= T;
+        block_sum2(&cnt, &ms, &sc, turn); turn ^= 1;
+        return cnt;
+    };
+
+    // ---- how many entries of E reach the threshold, how many the budget allows ---------------------------
+    int k_beta = m;
+    uint64_t T = ~0ull;                                  // keys <= T survive
+    bool have_T = false;
+    if (beta_ppm < 1000000ull && m > 0) {
+        const unsigned long long thr = ceil_muldiv(beta_ppm, total, 1000000ull);
+        if (thr == 0) k_beta = 1;
+        else {
+            T = search(thr, true);
+            k_beta = count_upto(T);
+            have_T = true;
+        }
     }
     int kc = k_beta;
     if (budget > 0) kc = min(kc, budget - (ln - m));
     kc = min(max(kc, 0), m);
+    if (kc < m && kc > 0 && !(have_T && kc == k_beta)) T = search((unsigned long long)kc, false);
 
-    for (int j = threadIdx.x; j < m; j += blockDim.x) flag[j] = 0;
-    __syncthreads();
-    for (int p = threadIdx.x; p < kc; p += blockDim.x) flag[(int)(uint32_t)keys[p]] = 1;
-    __syncthreads();
-
-    // ---- survivor map -----------------------------------------------------------------------
+    // ---- survivor map: my entries are consecutive, so a scan of the counts gives their places ------------------
     {
-        const int per = (m + blockDim.x - 1) / blockDim.x;
-        const int j0 = min(m, (int)threadIdx.x * per), j1 = min(m, j0 + per);
         int cnt = 0, first_drop = m;
-        for (int j = j0; j < j1; ++j) {
-            if (flag[j]) ++cnt; else if (first_drop == m) first_drop = j;
+#pragma unroll
+        for (int u = 0; u < KPT; ++u) {
+            if (j0 + u < m) {
+                const bool kept = kc >= m || (kc > 0 && key[u] <= T);
+                if (kept) ++cnt; else if (first_drop == m) first_drop = j0 + u;
+            }
         }
-        int total;
-        int off = block_exclusive_scan(cnt, scan_scratch, &total);
+        int tot;
+        int off = block_exclusive_scan(cnt, scan_scratch, &tot);
         if (first_drop < m) atomicMin(&s_first_drop, first_drop);
-        for (int j = j0; j < j1; ++j)
-            if (flag[j]) src[lo + off++] = lo + j;
+#pragma unroll
+        for (int u = 0; u < KPT; ++u)
+            if (j0 + u < m && (kc >= m || (kc > 0 && key[u] <= T))) {
+                src[lo + off] = lo + j0 + u;
+                an[lo + off] = acc[lo + j0 + u];
+                if (ps) pn[lo + off] = ps[lo + j0 + u];
+                ++off;
+            }
     }
     const int new_len = lo + kc + (ln - hi);
     for (int o = threadIdx.x; o < new_len; o += blockDim.x) {
         if (o < lo) src[o] = o;
-        else if (o >= lo + kc) src[o] = hi + (o - lo - kc);
+        else if (o >= lo + kc) {
+            const int sidx = hi + (o - lo - kc);
+            src[o] = sidx;
+            an[o] = acc[sidx];
+            if (ps) pn[o] = ps[sidx];
+        }
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -253,16 +238,162 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
         nout[m_idx] = new_len;
         len[m_idx] = new_len;
     }
-    // ---- per-entry arrays, in place, tiles in increasing order ---------------------------------
-    const int start = kc < m ? lo + s_first_drop : new_len;
-    int32_t* ps = pos ? pos + (int64_t)m_idx * cap : nullptr;
-    for (int o0 = start; o0 < new_len; o0 += blockDim.x) {
-        const int o = o0 + threadIdx.x;
-        float a = 0.f; int pv = 0;
-        __syncthreads();
-        if (o < new_len) { const int s = src[o]; a = acc[s]; if (ps) pv = ps[s]; }
-        __syncthreads();
-        if (o < new_len) { acc[o] = a; if (ps) ps[o] = pv; }
+}
+
+// The same for caches of up to 2048 rows: one WARP per (sequence, KV head), a lane holds KPL consecutive
+// entries, every sum is a handful of shuffles and no barrier is needed, so an SM works on dozens of heads at once.
+template <int KPL>
+__global__ void __launch_bounds__(128)
+kv_plan_warp_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __restrict__ e_lo,
+                    const int32_t* __restrict__ e_hi, int heads, int Hkv, int cap, int recent,
+                    unsigned long long beta_ppm, int budget, int32_t* __restrict__ src_map,
+                    int32_t* __restrict__ meta, int32_t* __restrict__ nout, float* __restrict__ acc_new,
+                    int32_t* __restrict__ pos_new, int32_t* dev_status) {
+    pdl_enter();
+    const int lane = threadIdx.x & 31;
+    const int m_idx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (m_idx >= heads) return;
+    const int b = m_idx / Hkv;
+    const int ln = len[m_idx];
+    int32_t* src = src_map + (int64_t)m_idx * cap;
+    float* acc = acc_score + (int64_t)m_idx * cap;
+    if (ln < 0 || ln > cap) {
+        if (lane == 0) {
+            if (dev_status) atomicOr(dev_status, LVLM_DEV_BOUNDS);
+            meta[m_idx] = 0; nout[m_idx] = 0;           // nothing moves, length left as it is
+        }
+        return;
+    }
+    int lo = e_lo ? e_lo[b] : 0;
+    int hi = e_hi ? e_hi[b] : ln;
+    hi = min(hi, ln - recent);
+    lo = min(max(lo, 0), ln);
+    hi = max(hi, lo);
+    const int m = hi - lo;
+
+    const int j0 = lane * KPL;
+    uint64_t key[KPL];
+    bool nonfinite = false;
+    uint64_t k_and = ~0ull, k_or = 0ull;
+    unsigned long long total = 0;
+#pragma unroll
+    for (int u = 0; u < KPL; ++u) {
+        key[u] = ~0ull;                                  // past the end: above every real key
+        if (j0 + u < m) {
+            const float sv = acc[lo + j0 + u];
+            key[u] = ((uint64_t)desc_key(sv, &nonfinite) << 32) | (uint32_t)(j0 + u);
+            k_and &= key[u]; k_or |= key[u];
+            total += (unsigned long long)score_units(sv);
+        }
+    }
+    if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        k_and &= __shfl_xor_sync(0xFFFFFFFFu, k_and, o);
+        k_or |= __shfl_xor_sync(0xFFFFFFFFu, k_or, o);
+        total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+    }
+    const uint64_t diff = m > 0 ? (k_and ^ k_or) : 0ull;
+    auto units_of = [](uint64_t k) -> unsigned long long {
+        const uint32_t dk = (uint32_t)(k >> 32);
+        if (dk == 0xFFFFFFFFu) return 0ull;
+        const uint32_t asc = ~dk;
+        const uint32_t bits = (asc & 0x80000000u) ? (asc & 0x7FFFFFFFu) : ~asc;
+        return (unsigned long long)score_units(__uint_as_float(bits));
+    };
+    auto search_count = [&](int target) -> uint64_t {
+        uint64_t ans = k_and, todo = diff;
+        while (todo) {
+            const int bit = 63 - __clzll((long long)todo);
+            todo &= ~(1ull << bit);
+            const uint64_t cand = (ans & ~(1ull << bit)) | ((1ull << bit) - 1ull);
+            int cnt = 0;
+#pragma unroll
+            for (int u = 0; u < KPL; ++u) cnt += key[u] <= cand;
+            cnt = warp_sum(cnt);
+            if (cnt >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
+        }
+        return ans;
+    };
+    auto search_mass = [&](unsigned long long target) -> uint64_t {
+        uint64_t ans = k_and, todo = diff;
+        while (todo) {
+            const int bit = 63 - __clzll((long long)todo);
+            todo &= ~(1ull << bit);
+            const uint64_t cand = (ans & ~(1ull << bit)) | ((1ull << bit) - 1ull);
+            unsigned long long ms = 0;
+#pragma unroll
+            for (int u = 0; u < KPL; ++u) if (key[u] <= cand) ms += units_of(key[u]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ms += __shfl_xor_sync(0xFFFFFFFFu, ms, o);
+            if (ms >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
+        }
+        return ans;
+    };
+
+    int k_beta = m;
+    uint64_t T = ~0ull;                                  // keys <= T survive
+    bool have_T = false;
+    if (beta_ppm < 1000000ull && m > 0) {
+        const unsigned long long thr = ceil_muldiv(beta_ppm, total, 1000000ull);
+        if (thr == 0) k_beta = 1;
+        else {
+            T = search_mass(thr);
+            int cnt = 0;
+#pragma unroll
+            for (int u = 0; u < KPL; ++u) cnt += key[u] <= T;
+            k_beta = warp_sum(cnt);
+            have_T = true;
+        }
+    }
+    int kc = k_beta;
+    if (budget > 0) kc = min(kc, budget - (ln - m));
+    kc = min(max(kc, 0), m);
+    if (kc < m && kc > 0 && !(have_T && kc == k_beta)) T = search_count(kc);
+
+    // survivor map: my entries are consecutive, so a scan of the counts over the lanes gives their places
+    int cnt = 0, first_drop = m;
+#pragma unroll
+    for (int u = 0; u < KPL; ++u) {
+        if (j0 + u < m) {
+            const bool kept = kc >= m || (kc > 0 && key[u] <= T);
+            if (kept) ++cnt; else if (first_drop == m) first_drop = j0 + u;
+        }
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    int off = incl - cnt;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first_drop = min(first_drop, __shfl_xor_sync(0xFFFFFFFFu, first_drop, o));
+    float* an = acc_new + (int64_t)m_idx * cap;
+    const int32_t* ps = pos ? pos + (int64_t)m_idx * cap : nullptr;
+    int32_t* pn = pos_new + (int64_t)m_idx * cap;
+#pragma unroll
+    for (int u = 0; u < KPL; ++u)
+        if (j0 + u < m && (kc >= m || (kc > 0 && key[u] <= T))) {
+            src[lo + off] = lo + j0 + u;
+            an[lo + off] = acc[lo + j0 + u];
+            if (ps) pn[lo + off] = ps[lo + j0 + u];
+            ++off;
+        }
+    const int new_len = lo + kc + (ln - hi);
+    for (int o = lane; o < new_len; o += 32) {
+        if (o < lo) src[o] = o;
+        else if (o >= lo + kc) {
+            const int sidx = hi + (o - lo - kc);
+            src[o] = sidx;
+            an[o] = acc[sidx];
+            if (ps) pn[o] = ps[sidx];
+        }
+    }
+    if (lane == 0) {
+        meta[m_idx] = kc < m ? lo + first_drop : new_len;
+        nout[m_idx] = new_len;
+        len[m_idx] = new_len;
     }
 }
 
@@ -287,25 +418,38 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
     int32_t* src_map = reinterpret_cast<int32_t*>(wsb + L.off_src);
     int32_t* meta = reinterpret_cast<int32_t*>(wsb + L.off_meta);
     int32_t* nout = reinterpret_cast<int32_t*>(wsb + L.off_nout);
+    float* acc_new = reinterpret_cast<float*>(wsb + L.off_acc);
+    int32_t* pos_new = reinterpret_cast<int32_t*>(wsb + L.off_pos);
 
     const unsigned long long beta_ppm = (unsigned long long)llrint((double)beta * 1.0e6);
-    const int P_max = next_pow2(d->cap < 2 ? 2 : d->cap);
-    int threads = P_max / 2;
-    threads = threads < 64 ? 64 : (threads > 1024 ? 1024 : threads);
-    const int binned = d->cap >= kPlanBinFrom && d->cap <= kPlanBinMaxCap;
-    const size_t smem = (size_t)P_max * 8 + (size_t)((d->cap + 1) & ~1) * 4 +
-                        (binned ? (size_t)P_max * 8 + (size_t)(2 * kPlanBins + 2) * 4 : 0);
-    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(kv_plan_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    {
-        const lvlm_status st = launch_kernel(kv_plan_kernel, dim3(d->Hkv, d->B), dim3(threads), smem, stream, 1,
-                                             acc_score, pos, len, e_lo, e_hi, d->Hkv, d->cap, d->recent, P_max, binned,
-                                             beta_ppm, budget, src_map, meta, nout, dev_status);
-        if (st != LVLM_OK) return st;
+    const int heads = d->B * d->Hkv;
+    lvlm_status st;
+#define LVLM_PLAN_WARP(KPL_)                                                                                     \
+    st = launch_kernel(kv_plan_warp_kernel<KPL_>, dim3((heads + 3) / 4), dim3(128), 0, stream, 1, acc_score, pos, len, \
+                       e_lo, e_hi, heads, d->Hkv, d->cap, d->recent, beta_ppm, budget, src_map, meta, nout, acc_new, pos_new, dev_status)
+    if (d->cap <= 512) LVLM_PLAN_WARP(16);
+    else if (d->cap <= 1024) LVLM_PLAN_WARP(32);
+    else if (d->cap <= 1536) LVLM_PLAN_WARP(48);
+    else if (d->cap <= 2048) LVLM_PLAN_WARP(64);
+    else {
+        // a CTA per head: a thread holds 4 entries (caches up to 4096 rows) or 16
+        const int kpt = d->cap <= 4096 ? 4 : 16;
+        int threads = ((d->cap + kpt - 1) / kpt + 31) / 32 * 32;
+        threads = threads < 64 ? 64 : threads;
+        st = kpt == 4 ? launch_kernel(kv_plan_kernel<4>, dim3(d->Hkv, d->B), dim3(threads), 0, stream, 1, acc_score, pos,
+                                      len, e_lo, e_hi, d->Hkv, d->cap, d->recent, beta_ppm, budget, src_map, meta, nout,
+                                      acc_new, pos_new, dev_status)
+                      : launch_kernel(kv_plan_kernel<16>, dim3(d->Hkv, d->B), dim3(threads), 0, stream, 1, acc_score, pos,
+                                      len, e_lo, e_hi, d->Hkv, d->cap, d->recent, beta_ppm, budget, src_map, meta, nout,
+                                      acc_new, pos_new, dev_status);
     }
+#undef LVLM_PLAN_WARP
+    if (st != LVLM_OK) return st;
     CompactJob j;
     j.base0 = Kc; j.base1 = Vc; j.stride_b = kv_sb * 2; j.stride_g = kv_sh * 2; j.B = d->B; j.G = d->Hkv;
     j.V = kHeadDim / 8; j.src_map = src_map; j.maps_per_g = d->Hkv; j.map_stride = d->cap;
     j.meta = meta; j.meta_stride = 1; j.nout = nout; j.N = d->cap;
+    j.side_dst[0] = acc_score; j.side_src[0] = acc_new;
+    if (pos) { j.side_dst[1] = pos; j.side_src[1] = pos_new; }
     return launch_inplace_compact(j, stream);
 }
