@@ -46,6 +46,14 @@ class LvlmError(RuntimeError):
 _lib = None
 
 
+def use_library(path: Optional[str]) -> None:
+    """Makes the binding load another build of the library at its next use (the tests load the build
+    with test hooks this way); None goes back to ``liblvlm.so``."""
+    global _lib, _LIB_PATH
+    _lib = None
+    _LIB_PATH = path or os.path.join(_PKG, "liblvlm.so")
+
+
 def lib() -> ctypes.CDLL:
     """The loaded library.  Raises if ``liblvlm.so`` has not been built (see build.py)."""
     global _lib
@@ -121,12 +129,6 @@ def _ws(ws, op, dims, device):
     if ws is None:
         ws = alloc_workspace(op, dims, device)
     return ws, ctypes.c_void_p(ws.data_ptr()), ctypes.c_size_t(ws.numel() * ws.element_size())
-
-
-def pyramid_schedule(n: int, final_ratio: float, stages: int):
-    """Image-token counts after each stage for a constant per-stage keep ratio that reaches
-    ``final_ratio`` after ``stages`` reductions (Appendix A.2)."""
-    return [int(math.floor(n * final_ratio ** (s / stages) + 0.5)) for s in range(1, stages + 1)]
 
 
 # ----------------------------------------------------------------------------------------------

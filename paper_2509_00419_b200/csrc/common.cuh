@@ -42,7 +42,7 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_launch_dependents(); }
 
-bool pdl_enabled();            // lvlm.cu; test hook lvlm_debug_set_pdl switches it off
+bool pdl_enabled();            // lvlm.cu: true, except in the test build when its hook switched it off
 
 // Launches `kernel` with programmatic stream serialisation and thread-block clusters of the given shape
 // (1, 1, 1 = no clusters).

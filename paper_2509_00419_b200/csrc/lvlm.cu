@@ -1,6 +1,4 @@
 // Version, status text and workspace sizes of the lvlm library.
-#include <cstdlib>
-
 #include "common.cuh"
 
 namespace lvlm {
@@ -10,16 +8,20 @@ size_t kv_compress_workspace(const lvlm_dims* d);
 size_t decode_attn_workspace(const lvlm_dims* d);
 }  // namespace lvlm
 
-// Programmatic dependent launch of the library's kernels: on unless the environment variable
-// LVLM_NO_PDL is set or the test hook below switches it off.  Not part of the public header.
-static int g_pdl = -1;
+// Programmatic dependent launch of the library's kernels is always on in the library proper.  The test build
+// (-DLVLM_TEST_HOOKS, a second shared object that only the tests load) can switch it off, to show that
+// no result depends on it.
+#ifdef LVLM_TEST_HOOKS
+static int g_pdl = 1;
 extern "C" void lvlm_debug_set_pdl(int on) { g_pdl = on ? 1 : 0; }
 namespace lvlm {
-bool pdl_enabled() {
-    if (g_pdl < 0) g_pdl = getenv("LVLM_NO_PDL") ? 0 : 1;
-    return g_pdl != 0;
-}
+bool pdl_enabled() { return g_pdl != 0; }
 }  // namespace lvlm
+#else
+namespace lvlm {
+bool pdl_enabled() { return true; }
+}  // namespace lvlm
+#endif
 
 extern "C" const char* lvlm_version(void) { return "lvlm 0.1 (sm_100a)"; }
 

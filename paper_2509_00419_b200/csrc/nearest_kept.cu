@@ -503,12 +503,14 @@ nk_sim_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ 
             tc_fence_before();
             mbar_arrive(&sm->tmem_empty[buf]);
         }
-        // the two column halves of a row meet in shared memory (the lower half holds the lower indices
-        // and wins ties); every epilogue thread comes here, also after a timeout
+        // the two column halves of a row meet in shared memory (on equal similarity the lower kept index
+        // wins, whichever half and column tile it sits in); every epilogue thread comes here, also after a timeout
         if (half == 1) { sm->xv[row] = best_v; sm->xt[row] = best_t; }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (half == 0) {
-            if (sm->xt[row] >= 0 && (best_t < 0 || sm->xv[row] > best_v)) { best_v = sm->xv[row]; best_t = sm->xt[row]; }
+            const float ov = sm->xv[row];
+            const int ot = sm->xt[row];
+            if (ot >= 0 && (best_t < 0 || ov > best_v || (ov == best_v && ot < best_t))) { best_v = ov; best_t = ot; }
             const int q = rt * kSimM + row;
             if (!sm->abort && q < a.r && best_t >= 0) {
                 uint32_t u = __float_as_uint(best_v);

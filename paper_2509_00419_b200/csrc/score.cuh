@@ -9,10 +9,6 @@ struct ScoreStrides { int64_t q_sb, q_sn, q_sh, kv_sb, kv_sh; };   // elements
 
 bool score_layout(const lvlm_dims* d, ScoreLayout* L);
 
-lvlm_status launch_score_reduce(const float* partial, bool group_summed, const lvlm_dims* d,
-                                float* score, float* score_head, int32_t* dev_status,
-                                cudaStream_t stream);
-
 // Tensor-core path: pass 1 (row normalisers into lse_ws, skipped when the caller supplies lse) and
 // pass 2 (column sums per CTA row into partial, added over the heads by the last CTA of each key
 // tile, which writes score and score_head).  cnt holds one counter per (sequence, key tile).

@@ -5,12 +5,19 @@ library's kernels.  Used by the benchmark and by the full-size parity tests.
 """
 from __future__ import annotations
 
+import math
 from typing import List, Optional
 
 import torch
 
 from . import binding as L
 from . import inputs as I
+
+
+def pyramid_schedule(n: int, final_ratio: float, stages: int):
+    """Image-token counts after each stage for a constant per-stage keep ratio that reaches
+    ``final_ratio`` after ``stages`` reductions (Appendix A.2).  The library itself receives integers."""
+    return [int(math.floor(n * final_ratio ** (s / stages) + 0.5)) for s in range(1, stages + 1)]
 
 
 class ReduceStage:

@@ -71,32 +71,43 @@ def _check_pyramid(w, sample):
     return near_ties
 
 
+def _report_near_ties(w, sample, near_ties):
+    """Rank disagreements are accepted only as swaps of near-tied tokens (checked one by one above); their
+    number is reported and has to stay a negligible share of the tokens ranked."""
+    ranked = len(sample) * sum([w.n] + [m for _, m in w.stages[:-1]])
+    print(f"{w.name}: {near_ties} near-tie rank swaps among {ranked} ranked tokens of the sampled sequences")
+    assert near_ties <= max(2, ranked // 200)            # 0.5 %: with 16384 tokens many scores lie within 1e-4 of a neighbour
+
+
 def test_cfg2_pyramid_full_size():
-    _check_pyramid(I.CFG2, sample=[0])
+    _report_near_ties(I.CFG2, [0], _check_pyramid(I.CFG2, sample=[0]))
 
 
 def test_cfg2_alt_schedule_full_size():
-    _check_pyramid(I.CFG2_ALT, sample=[0])
+    _report_near_ties(I.CFG2_ALT, [0], _check_pyramid(I.CFG2_ALT, sample=[0]))
 
 
 def test_cfg3_batched_prefill_full_size():
-    _check_pyramid(I.CFG3, sample=[0, 11])
+    _report_near_ties(I.CFG3, [0, 11], _check_pyramid(I.CFG3, sample=[0, 11]))
 
 
 def test_cfg5_extreme_reduction_full_size():
-    _check_pyramid(I.CFG5, sample=[0])
+    _report_near_ties(I.CFG5, [0], _check_pyramid(I.CFG5, sample=[0]))
 
 
 def test_video_length_pyramid_full_size():
     """32768 image tokens (64 frames): the second workload shape the paper evaluates (video benchmarks)."""
-    _check_pyramid(I.VIDEO, sample=[0])
+    _report_near_ties(I.VIDEO, [0], _check_pyramid(I.VIDEO, sample=[0]))
 
 
-def _decode_chunks(w, n_layers, prompt_len, steps, check_steps, dev):
+def _decode_chunks(w, n_layers, prompt_len, steps, check_at, dev, check_layers=None):
     """Decode loop with the periodic budgeted compression at the workload's full batch and head
     counts, on ``n_layers`` layers.  The oracle restarts from a copy of the GPU state at the start of
     every chunk of ``trigger`` steps (so that a near-tie in an eviction cannot cascade), redoes the
-    compression bit-exactly on the GPU's own scores and follows the first ``check_steps`` steps."""
+    compression bit-exactly on the GPU's own scores, and checks the steps of the chunk listed in
+    ``check_at`` (offsets inside the chunk; before a step that does not follow a checked one it takes
+    a fresh copy of the GPU state), on the layers ``check_layers`` (default: all)."""
+    check_layers = list(range(n_layers)) if check_layers is None else check_layers
     dec = P.DecodeLayers(n_layers, w.B, w.H, w.Hkv, w.cap, dev)
     pos = torch.arange(prompt_len, dtype=torch.int32, device=dev)[None].repeat(w.B, 1) % w.N
     T = min(w.T, prompt_len)
@@ -115,12 +126,14 @@ def _decode_chunks(w, n_layers, prompt_len, steps, check_steps, dev):
         ns = min(w.trigger, steps - c0)
         qs, ks, vs = zip(*[I.decode_inputs(w, l, c0, ns, dev) for l in range(n_layers)])
         qs, ks, vs = torch.stack(qs, 1), torch.stack(ks, 1), torch.stack(vs, 1)      # [ns, layers, ...]
-        state = [dict(K=f64(dec.K[l]), V=f64(dec.V[l]), acc=dec.acc[l].cpu().numpy().copy(),
-                      len=i32(dec.len[l])) for l in range(n_layers)]
+        snap = lambda l: dict(K=f64(dec.K[l]), V=f64(dec.V[l]), acc=dec.acc[l].cpu().numpy().copy(),
+                              len=i32(dec.len[l]))
+        state = {l: snap(l) for l in check_layers}
+        fresh = True                                  # the oracle state equals the GPU state right now
         if cur > w.budget:
             dec.compress(beta=1.0, budget=w.budget, recent=w.recent)
             compressions += 1
-            for l in range(n_layers):
+            for l in check_layers:
                 o = O.kv_compress(state[l]["K"], state[l]["V"], state[l]["acc"], state[l]["len"],
                                   beta=1.0, budget=w.budget, recent=w.recent)
                 m = w.budget
@@ -132,10 +145,14 @@ def _decode_chunks(w, n_layers, prompt_len, steps, check_steps, dev):
                                 acc=o["acc_score"], len=o["len"])
             cur = w.budget
         for t in range(ns):
+            if t in check_at and not fresh:
+                torch.cuda.synchronize()
+                state = {l: snap(l) for l in check_layers}
             dec.decode_step(qs[t], ks[t], vs[t], accumulate=True)
             cur += 1
-            if t < check_steps:
-                for l in range(n_layers):
+            fresh = t in check_at
+            if t in check_at:
+                for l in check_layers:
                     o = O.decode_attn(f64(qs[t, l]), state[l]["K"], state[l]["V"], state[l]["len"],
                                       k_new=f64(ks[t, l]), v_new=f64(vs[t, l]), acc_score=state[l]["acc"])
                     assert_rows_close(f64(dec.out[l]), o["out"], what=f"step {c0 + t} layer {l} output")
@@ -150,15 +167,27 @@ def _decode_chunks(w, n_layers, prompt_len, steps, check_steps, dev):
 
 
 def test_cfg4_long_decode_with_periodic_compression():
+    """Two layers over the whole 4096-step generation; the oracle follows the first two steps of every chunk of
+    128 and one step in its middle."""
     w = I.CFG4
-    n = _decode_chunks(w, n_layers=2, prompt_len=w.N, steps=1024, check_steps=2, dev=torch.device("cuda", 0))
-    assert n == 4          # 640 -> 1152 after 512 steps, then every 128 steps
+    n = _decode_chunks(w, n_layers=2, prompt_len=w.N, steps=w.decode_steps, check_at=(0, 1, 77),
+                       dev=torch.device("cuda", 0))
+    assert n == 28         # 640 -> 1152 after 512 steps, then every 128 steps
+
+
+def test_cfg4_all_layers_decode_with_compression():
+    """All 32 layers for 256 steps from a cache that is about to overflow (a compression at the second chunk);
+    the oracle follows six of the layers, lengths and status are checked on all."""
+    w = I.CFG4
+    n = _decode_chunks(w, n_layers=w.L, prompt_len=1000, steps=256, check_at=(0, 100),
+                       dev=torch.device("cuda", 0), check_layers=[0, 1, 9, 17, 30, 31])
+    assert n == 1
 
 
 def test_cfg5_decode_after_extreme_reduction():
     w = I.CFG5
     prompt = w.stages[-1][1] + w.T + w.i0
-    n = _decode_chunks(w, n_layers=2, prompt_len=prompt, steps=384, check_steps=2, dev=torch.device("cuda", 0))
+    n = _decode_chunks(w, n_layers=2, prompt_len=prompt, steps=384, check_at=(0, 1, 50), dev=torch.device("cuda", 0))
     assert n == 3          # 748 entries after prefill: every chunk starts above the budget of 512
 
 

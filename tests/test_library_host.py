@@ -120,6 +120,7 @@ def test_binding_refuses_cpu_tensors():
 
 
 def test_schedule_host_function():
-    assert L.pyramid_schedule(2880, 0.03, 3) == [895, 278, 86]
-    assert L.pyramid_schedule(1792, 0.35, 2) == [1060, 627]
+    from paper_2509_00419_b200 import pipeline as P
+    assert P.pyramid_schedule(2880, 0.03, 3) == [895, 278, 86]
+    assert P.pyramid_schedule(1792, 0.35, 2) == [1060, 627]
     assert L.merged_rows(640, 576, 287) == 352 and L.merged_rows(640, 576, 576) == 640

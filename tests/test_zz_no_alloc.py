@@ -3,7 +3,7 @@ device memory (a plug-in inside an engine that owns the whole memory pool, a bin
 ever sees raw pointers, a loop that must not meet cudaMalloc's device-wide synchronisation).
 
 It keeps its scratch in a fixed array inside the library, so the checks that matter are: it gives
-what lvlm_decode_attn gives, it still does so on a second call that finds the first call's
+what lvlm_decode_attn gives (and what the oracle gives), it still does so on a later call that finds the first call's
 leftovers in the array, it allocates nothing, and it refuses problems that do not fit.
 
 This file sorts after every other test file on purpose: a run that stops at the first failure has
@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import lvlm_oracle as O
 from paper_2509_00419_b200 import binding as L
 from paper_2509_00419_b200 import build as B
 from util import assert_rows_close, assert_scores_close, f64
@@ -34,11 +35,14 @@ def _case(seed, Bq, H, Hkv, cap, device):
 def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row():
     B.build()
     dev = torch.device("cuda", 0)
-    # two different problems back to back: the second one finds the first one's partial results,
-    # split layout and logits still sitting in the shared array
-    for seed, (Bq, H, Hkv, cap) in enumerate([(2, 32, 8, 1152), (3, 28, 4, 300)]):
+    # different problems back to back: each one finds the leftovers of the one before in the shared array.  The
+    # last one has runs of keys too long for a CTA's logits to stay in shared memory, so it is the one that
+    # really parks them in the array.
+    for seed, (Bq, H, Hkv, cap) in enumerate([(2, 32, 8, 1152), (3, 28, 4, 300), (1, 8, 1, 8192)]):
         c = _case(seed, Bq, H, Hkv, cap, dev)
         ref = {k: v.clone() for k, v in c.items()}
+        truth = O.decode_attn(f64(c["q"]), f64(c["K"]), f64(c["V"]), c["ln"].cpu().numpy(), k_new=f64(c["kn"]),
+                              v_new=f64(c["vn"]), acc_score=c["acc"].cpu().numpy().copy())
         want = L.decode_attn(ref["q"], ref["K"], ref["V"], ref["ln"], k_new=ref["kn"], v_new=ref["vn"],
                              acc_score=ref["acc"])
         out = torch.empty_like(c["q"])
@@ -52,12 +56,16 @@ def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row():
         assert allocations() == before                   # torch's allocator was not asked for anything
         assert got.data_ptr() == out.data_ptr() and flag.item() == 0
         assert_rows_close(f64(got), f64(want), what=f"call {seed}: attention output")
+        assert_rows_close(f64(got), truth["out"], what=f"call {seed}: attention output against the oracle")
+        assert np.array_equal(c["ln"].cpu().numpy(), truth["len"])
         assert torch.equal(c["ln"], ref["ln"]) and torch.equal(c["K"], ref["K"]) and torch.equal(c["V"], ref["V"])
         for b in range(Bq):
             for g in range(Hkv):
                 m = int(c["ln"][b, g])
                 assert_scores_close(c["acc"][b, g, :m].cpu().numpy(), ref["acc"][b, g, :m].cpu().numpy(),
                                     what=f"call {seed}: acc_score")
+                assert_scores_close(c["acc"][b, g, :m].cpu().numpy(), truth["acc_score"][b, g, :m],
+                                    what=f"call {seed}: acc_score against the oracle")
 
 
 @pytest.mark.gpu
