@@ -33,7 +33,6 @@ constexpr int kBoxBytes = kStageKeys * 128;          // one TMA box: 64 keys x 6
 constexpr int kStageBytes = 4 * kBoxBytes;           // K low half, K high half, V low half, V high half
 constexpr int kStagesDec = 3;
 constexpr int kRingBytes = kStagesDec * kStageBytes;
-constexpr int kDecAccFloats = 2048;                  // shared floats for merging the warps of a CTA (8 KB)
 constexpr int kDecTargetCtas = 2 * 148;              // CTAs wanted in flight: two per SM of a 148-SM part
 constexpr int kDecMaxCluster = 8;                    // portable cluster size
 constexpr int kDecMinTiles = 2;                      // a CTA's run is not made shorter than this by splitting

@@ -52,9 +52,10 @@ __device__ __forceinline__ unsigned long long ceil_muldiv(unsigned long long a, 
     return q + (rem != 0);
 }
 
-// Sums over the block of a count and a 64-bit mass (one barrier: the scratch rows alternate with `turn`).
+// Sums over the first `nwarp` warps of the block of a count and a 64-bit mass (one barrier: the scratch rows
+// alternate with `turn`).
 struct PlanScratch { int c[2][32]; unsigned long long m[2][32]; };
-__device__ __forceinline__ void block_sum2(int* c, unsigned long long* ms, PlanScratch* sc, int turn) {
+__device__ __forceinline__ void block_sum2(int* c, unsigned long long* ms, PlanScratch* sc, int turn, int nwarp) {
     int cc = *c;
     unsigned long long mm = *ms;
 #pragma unroll
@@ -62,9 +63,9 @@ __device__ __forceinline__ void block_sum2(int* c, unsigned long long* ms, PlanS
         cc += __shfl_xor_sync(0xFFFFFFFFu, cc, o);
         mm += __shfl_xor_sync(0xFFFFFFFFu, mm, o);
     }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (lane == 0) { sc->c[turn][warp] = cc; sc->m[turn][warp] = mm; }
-    __syncthreads();
+    asm volatile("bar.sync 1, %0;" ::"r"(nwarp * 32) : "memory");       // the warps that hold entries
     cc = 0; mm = 0;
     for (int wv = 0; wv < nwarp; ++wv) { cc += sc->c[turn][wv]; mm += sc->m[turn][wv]; }
     *c = cc; *ms = mm;
@@ -79,7 +80,7 @@ __device__ __forceinline__ void block_sum2(int* c, unsigned long long* ms, PlanS
 template <int KPT>
 __global__ void __launch_bounds__(1024)
 kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __restrict__ e_lo,
-               const int32_t* __restrict__ e_hi, int Hkv, int cap, int recent,
+               const int32_t* __restrict__ e_hi, int Hkv, int cap, int recent, int min_m,
                unsigned long long beta_ppm, int budget, int32_t* __restrict__ src_map,
                int32_t* __restrict__ meta, int32_t* __restrict__ nout, float* __restrict__ acc_new,
                int32_t* __restrict__ pos_new, int32_t* dev_status) {
@@ -107,6 +108,11 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
     lo = min(max(lo, 0), ln);
     hi = max(hi, lo);
     const int m = hi - lo;
+    if (m < min_m) return;                               // a head this small was planned by the warp kernel
+    // only the warps that hold entries stay: every barrier below counts them alone
+    const int nwarp = max(1, (m + 32 * KPT - 1) / (32 * KPT)), nthr = nwarp * 32;
+    if ((int)threadIdx.x >= nthr) return;
+    auto sync_active = [&]() { asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory"); };
     if (threadIdx.x == 0) s_first_drop = m;
     // compacted acc_score and pos go beside the map; the kernel that moves the K and V rows copies them back
     float* an = acc_new + (int64_t)m_idx * cap;
@@ -116,6 +122,7 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
     // ---- my keys -------------------------------------------------------------------------------------
     const int j0 = threadIdx.x * KPT;
     uint64_t key[KPT];
+    unsigned long long un[KPT];                          // the scores in integer units
     bool nonfinite = false;
     uint64_t k_and = ~0ull, k_or = 0ull;
     unsigned long long total = 0;
@@ -123,22 +130,16 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
 #pragma unroll
     for (int u = 0; u < KPT; ++u) {
         key[u] = ~0ull;                                  // past the end: above every real key
+        un[u] = 0ull;
         if (j0 + u < m) {
             const float sv = acc[lo + j0 + u];
             key[u] = ((uint64_t)desc_key(sv, &nonfinite) << 32) | (uint32_t)(j0 + u);
             k_and &= key[u]; k_or |= key[u];
-            total += (unsigned long long)score_units(sv);
+            un[u] = (unsigned long long)score_units(sv);
+            total += un[u];
         }
     }
     if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
-    // units of a key's score, recomputed from the key when a sum needs them
-    auto units_of = [](uint64_t k) -> unsigned long long {
-        const uint32_t dk = (uint32_t)(k >> 32);
-        if (dk == 0xFFFFFFFFu) return 0ull;             // NaN (or no entry)
-        const uint32_t asc = ~dk;
-        const uint32_t bits = (asc & 0x80000000u) ? (asc & 0x7FFFFFFFu) : ~asc;
-        return (unsigned long long)score_units(__uint_as_float(bits));
-    };
     {   // bits in which the keys differ, and the total score
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -147,9 +148,9 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
         }
         if ((threadIdx.x & 31) == 0) { s_and[threadIdx.x >> 5] = k_and; s_or[threadIdx.x >> 5] = k_or; }
         int dummy = 0;
-        block_sum2(&dummy, &total, &sc, turn); turn ^= 1;            // (its barrier also publishes s_and / s_or)
+        block_sum2(&dummy, &total, &sc, turn, nwarp); turn ^= 1;            // (its barrier also publishes s_and / s_or)
         k_and = ~0ull; k_or = 0ull;
-        for (int wv = 0; wv < (int)(blockDim.x >> 5); ++wv) { k_and &= s_and[wv]; k_or |= s_or[wv]; }
+        for (int wv = 0; wv < nwarp; ++wv) { k_and &= s_and[wv]; k_or |= s_or[wv]; }
     }
     const uint64_t diff = m > 0 ? (k_and ^ k_or) : 0ull;
     // Smallest key T such that the entries with key <= T hold at least `target` (their count, or their score when
@@ -165,9 +166,9 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
             unsigned long long ms = 0;
 #pragma unroll
             for (int u = 0; u < KPT; ++u) {
-                if (key[u] <= cand) { ++cnt; if (by_mass) ms += units_of(key[u]); }
+                if (key[u] <= cand) { ++cnt; ms += un[u]; }
             }
-            block_sum2(&cnt, &ms, &sc, turn); turn ^= 1;
+            block_sum2(&cnt, &ms, &sc, turn, nwarp); turn ^= 1;
             const unsigned long long have = by_mass ? ms : (unsigned long long)cnt;
             if (have >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
         }
@@ -178,7 +179,7 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
         unsigned long long ms = 0;
 #pragma unroll
         for (int u = 0; u < KPT; ++u) cnt += key[u] <= T;
-        block_sum2(&cnt, &ms, &sc, turn); turn ^= 1;
+        block_sum2(&cnt, &ms, &sc, turn, nwarp); turn ^= 1;
         return cnt;
     };
 
@@ -210,8 +211,18 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
                 if (kept) ++cnt; else if (first_drop == m) first_drop = j0 + u;
             }
         }
-        int tot;
-        int off = block_exclusive_scan(cnt, scan_scratch, &tot);
+        // exclusive scan of the counts over the active warps
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) scan_scratch[warp] = incl;
+        sync_active();
+        int off = incl - cnt;
+        for (int wv = 0; wv < warp; ++wv) off += scan_scratch[wv];
         if (first_drop < m) atomicMin(&s_first_drop, first_drop);
 #pragma unroll
         for (int u = 0; u < KPT; ++u)
@@ -223,7 +234,7 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
             }
     }
     const int new_len = lo + kc + (ln - hi);
-    for (int o = threadIdx.x; o < new_len; o += blockDim.x) {
+    for (int o = threadIdx.x; o < new_len; o += nthr) {
         if (o < lo) src[o] = o;
         else if (o >= lo + kc) {
             const int sidx = hi + (o - lo - kc);
@@ -232,7 +243,7 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
             if (ps) pn[o] = ps[sidx];
         }
     }
-    __syncthreads();
+    sync_active();
     if (threadIdx.x == 0) {
         meta[m_idx] = kc < m ? lo + s_first_drop : new_len;
         nout[m_idx] = new_len;
@@ -245,7 +256,7 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
 template <int KPL>
 __global__ void __launch_bounds__(128)
 kv_plan_warp_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __restrict__ e_lo,
-                    const int32_t* __restrict__ e_hi, int heads, int Hkv, int cap, int recent,
+                    const int32_t* __restrict__ e_hi, int heads, int Hkv, int cap, int recent, int only_small,
                     unsigned long long beta_ppm, int budget, int32_t* __restrict__ src_map,
                     int32_t* __restrict__ meta, int32_t* __restrict__ nout, float* __restrict__ acc_new,
                     int32_t* __restrict__ pos_new, int32_t* dev_status) {
@@ -270,20 +281,26 @@ kv_plan_warp_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t*
     lo = min(max(lo, 0), ln);
     hi = max(hi, lo);
     const int m = hi - lo;
+    if (only_small && m > 32 * KPL) return;              // too many entries for the registers: the CTA kernel plans it
 
     const int j0 = lane * KPL;
     uint64_t key[KPL];
+    constexpr bool kKeepUnits = KPL <= 32;               // the scores in integer units stay in registers when they fit
+    unsigned long long un[kKeepUnits ? KPL : 1];
     bool nonfinite = false;
     uint64_t k_and = ~0ull, k_or = 0ull;
     unsigned long long total = 0;
 #pragma unroll
     for (int u = 0; u < KPL; ++u) {
         key[u] = ~0ull;                                  // past the end: above every real key
+        if (kKeepUnits) un[u] = 0ull;
         if (j0 + u < m) {
             const float sv = acc[lo + j0 + u];
             key[u] = ((uint64_t)desc_key(sv, &nonfinite) << 32) | (uint32_t)(j0 + u);
             k_and &= key[u]; k_or |= key[u];
-            total += (unsigned long long)score_units(sv);
+            const unsigned long long su = (unsigned long long)score_units(sv);
+            if (kKeepUnits) un[u] = su;
+            total += su;
         }
     }
     if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
@@ -323,7 +340,7 @@ kv_plan_warp_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t*
             const uint64_t cand = (ans & ~(1ull << bit)) | ((1ull << bit) - 1ull);
             unsigned long long ms = 0;
 #pragma unroll
-            for (int u = 0; u < KPL; ++u) if (key[u] <= cand) ms += units_of(key[u]);
+            for (int u = 0; u < KPL; ++u) if (key[u] <= cand) ms += kKeepUnits ? un[u] : units_of(key[u]);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) ms += __shfl_xor_sync(0xFFFFFFFFu, ms, o);
             if (ms >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
@@ -424,24 +441,34 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
     const unsigned long long beta_ppm = (unsigned long long)llrint((double)beta * 1.0e6);
     const int heads = d->B * d->Hkv;
     lvlm_status st;
-#define LVLM_PLAN_WARP(KPL_)                                                                                     \
+#define LVLM_PLAN_WARP(KPL_, SMALL_)                                                                             \
     st = launch_kernel(kv_plan_warp_kernel<KPL_>, dim3((heads + 3) / 4), dim3(128), 0, stream, 1, acc_score, pos, len, \
-                       e_lo, e_hi, heads, d->Hkv, d->cap, d->recent, beta_ppm, budget, src_map, meta, nout, acc_new, pos_new, dev_status)
-    if (d->cap <= 512) LVLM_PLAN_WARP(16);
-    else if (d->cap <= 1024) LVLM_PLAN_WARP(32);
-    else if (d->cap <= 1536) LVLM_PLAN_WARP(48);
-    else if (d->cap <= 2048) LVLM_PLAN_WARP(64);
-    else {
-        // a CTA per head: a thread holds 4 entries (caches up to 4096 rows) or 16
-        const int kpt = d->cap <= 4096 ? 4 : 16;
-        int threads = ((d->cap + kpt - 1) / kpt + 31) / 32 * 32;
-        threads = threads < 64 ? 64 : threads;
+                       e_lo, e_hi, heads, d->Hkv, d->cap, d->recent, SMALL_, beta_ppm, budget, src_map, meta, nout,   \
+                       acc_new, pos_new, dev_status)
+    const bool many = heads >= 4 * 148;                 // enough heads to fill the GPU with one warp each
+    const int kpt = d->cap <= 4096 ? 4 : 16;
+    int threads = ((d->cap + kpt - 1) / kpt + 31) / 32 * 32;
+    threads = threads < 64 ? 64 : threads;
+    int min_m = 0;                                       // heads the CTA kernel leaves to the warp kernel
+    bool cta_kernel = true;
+    if (many) {
+        if (d->cap <= 512) LVLM_PLAN_WARP(16, 0);
+        else if (d->cap <= 1024) LVLM_PLAN_WARP(32, 0);
+        else if (d->cap <= 1536) LVLM_PLAN_WARP(48, 0);
+        else if (d->cap <= 2048) LVLM_PLAN_WARP(64, 0);
+        else LVLM_PLAN_WARP(32, 1);                      // long caches: the heads with up to 1024 evictable entries
+        if (st != LVLM_OK) return st;
+        cta_kernel = d->cap > 2048;                      // ... the others get a CTA each
+        min_m = 32 * 32 + 1;
+    }
+    if (cta_kernel) {
+        // a CTA per head, a thread holds 4 entries (caches up to 4096 rows) or 16; warps without entries leave at once
         st = kpt == 4 ? launch_kernel(kv_plan_kernel<4>, dim3(d->Hkv, d->B), dim3(threads), 0, stream, 1, acc_score, pos,
-                                      len, e_lo, e_hi, d->Hkv, d->cap, d->recent, beta_ppm, budget, src_map, meta, nout,
-                                      acc_new, pos_new, dev_status)
+                                      len, e_lo, e_hi, d->Hkv, d->cap, d->recent, min_m, beta_ppm, budget, src_map,
+                                      meta, nout, acc_new, pos_new, dev_status)
                       : launch_kernel(kv_plan_kernel<16>, dim3(d->Hkv, d->B), dim3(threads), 0, stream, 1, acc_score, pos,
-                                      len, e_lo, e_hi, d->Hkv, d->cap, d->recent, beta_ppm, budget, src_map, meta, nout,
-                                      acc_new, pos_new, dev_status);
+                                      len, e_lo, e_hi, d->Hkv, d->cap, d->recent, min_m, beta_ppm, budget, src_map,
+                                      meta, nout, acc_new, pos_new, dev_status);
     }
 #undef LVLM_PLAN_WARP
     if (st != LVLM_OK) return st;
