@@ -11,6 +11,7 @@ Steps, in the paper's order and notation (Section 3.2.1 pyramid token merging,
 Section 3.2.2 KV-cache compression, Appendix A.2 settings):
 
   score_tokens    per-key summed attention A, head-averaged        Sec. 3.2.1 par. 3
+  attention_with_scores  the layer's attention itself, returning A  Sec. 3.2.1 par. 3 + footnote
   select_topk     split into P_unmerged / P_merged by A, ordered   Sec. 3.2.1 par. 4
   merge_weights   the weight list W_v                              Sec. 3.2.1 par. 4
   merge_compact   P_new = W_v x P_merged; P_compressed             Sec. 3.2.1 par. 4
@@ -20,7 +21,9 @@ Section 3.2.2 KV-cache compression, Appendix A.2 settings):
   pyramid_schedule constant reduction ratio from the final budget  App. A.2
 
 Pins (tests/test_oracle_pins.py): textbook softmax, row-sum and harmonic-number
-closed forms for the score; brute-force subset enumeration for the selection;
+closed forms for the score; for attention_with_scores its last row against
+decode_attn, its column sums against score_tokens, row sums of one and
+scipy's logsumexp; brute-force subset enumeration for the selection;
 closed-form weights, literal iterated pairwise merging and identities for the
 merge; no-op / arg-max / uniform-count closed forms for the compression;
 len-1, equal-key and GQA identities for decode attention; the printed stage
@@ -94,6 +97,48 @@ def score_tokens(Q, K, q_lo, q_hi, i0, n, causal=True, scale=None):
     score = s_head.mean(axis=1)
     score_head = s_head.reshape(B, Hkv, G, n).sum(axis=2)
     return score.astype(np.float32), score_head.astype(np.float32)
+
+
+def attention_with_scores(Q, K, V, q_lo, q_hi, i0, n, causal=True, scale=None):
+    """The attention of a prefill layer, returning alongside its output what the token
+    reduction reads from it (Section 3.2.1, paragraph 3 and its footnote: the per-key summed
+    scores are a by-product of the attention that runs anyway).
+
+    Q  [B, N, H, D]   query rows of sequence positions 0..N-1
+    K, V [B, Hkv, N, D]
+    Row p attends with softmax over the keys it sees (j <= p when causal).  Returns a dict:
+      out        [B, N, H, D] bf16-rounded float32: softmax(Q K^T scale) V
+      lse        [B, H, N]    float32: natural log of each row's sum of exponentials
+      score      [B, n], score_head [B, Hkv, n]  float32: the probabilities of the rows
+                 q_lo..q_hi-1 summed per image key j in [i0, i0+n), head mean / group sum
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    B, N, H, D = Q.shape
+    Hkv = K.shape[1]
+    assert K.shape[2] == N and V.shape[:3] == K.shape[:3] and H % Hkv == 0 and 0 <= q_lo < q_hi <= N
+    G = H // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    visible = (np.arange(N)[None, :] <= np.arange(N)[:, None]) if causal else np.ones((N, N), bool)
+    out = np.zeros((B, N, H, V.shape[3]))
+    lse = np.zeros((B, H, N))
+    s_head = np.zeros((B, H, n))
+    for b in range(B):
+        for h in range(H):
+            logits = (Q[b, :, h, :] @ K[b, h // G].T) * scale            # [N, N]
+            logits = np.where(visible, logits, -np.inf)
+            m = logits.max(axis=1, keepdims=True)
+            e = np.exp(logits - m)
+            z = e.sum(axis=1, keepdims=True)
+            p = e / z
+            out[b, :, h, :] = p @ V[b, h // G]
+            lse[b, h] = (m + np.log(z))[:, 0]
+            s_head[b, h] = p[q_lo:q_hi, i0:i0 + n].sum(axis=0)
+    return {"out": round_bf16(out), "lse": lse.astype(np.float32),
+            "score": s_head.mean(axis=1).astype(np.float32),
+            "score_head": s_head.reshape(B, Hkv, G, n).sum(axis=2).astype(np.float32)}
 
 
 # ----------------------------------------------------------------------------

@@ -408,6 +408,48 @@ def test_kv_evictable_range_budget_and_recent_window():
 
 
 # ------------------------------------------------------------------ decode attention
+# ------------------------------------------------------------------ attention_with_scores
+def _bf(r, *shape):
+    return O.round_bf16(r.normal(size=shape)).astype(np.float64)
+
+
+def test_attention_last_row_is_decode_attention_and_rows_sum_to_one():
+    r = np.random.default_rng(21)
+    B, N, H, Hkv, D = 2, 37, 6, 2, 16
+    Q, K, V = _bf(r, B, N, H, D), _bf(r, B, Hkv, N, D), _bf(r, B, Hkv, N, D)
+    a = O.attention_with_scores(Q, K, V, 30, N, 3, 20)
+    # the last position sees every key: its output is one decode step over the whole cache
+    dec = O.decode_attn(Q[:, N - 1], K, V, np.full((B, Hkv), N, np.int32))
+    assert np.array_equal(a["out"][:, N - 1], dec["out"])
+    # every position p is a decode step over the first p+1 entries
+    for p in (0, 1, 17):
+        dec = O.decode_attn(Q[:, p], K, V, np.full((B, Hkv), p + 1, np.int32))
+        assert np.array_equal(a["out"][:, p], dec["out"])
+    # lse is the log of the row's sum of exponentials (library routine), so exp(logit - lse) sums to one
+    scale = 1.0 / math.sqrt(D)
+    for b, h, p in [(0, 0, 0), (1, 5, 36), (0, 3, 12)]:
+        logits = (Q[b, p, h] @ K[b, h // 3, :p + 1].T) * scale
+        assert abs(a["lse"][b, h, p] - scipy.special.logsumexp(logits)) < 1e-5
+        assert abs(np.exp(logits - a["lse"][b, h, p].astype(np.float64)).sum() - 1.0) < 1e-5
+
+
+def test_attention_column_sums_are_the_scores_of_the_window():
+    r = np.random.default_rng(22)
+    B, N, H, Hkv, D = 1, 50, 4, 2, 8
+    Q, K, V = _bf(r, B, N, H, D), _bf(r, B, Hkv, N, D), _bf(r, B, Hkv, N, D)
+    for (q_lo, q_hi, i0, n) in [(40, 50, 2, 35), (0, 50, 0, 50), (10, 11, 5, 4)]:
+        a = O.attention_with_scores(Q, K, V, q_lo, q_hi, i0, n)
+        score, head = O.score_tokens(Q[:, q_lo:q_hi], K, q_lo, q_hi, i0, n)
+        assert np.array_equal(a["score"], score) and np.array_equal(a["score_head"], head)
+    # a transposed operand or a dropped mask shows here: V = identity-like rows give the probabilities back
+    Vp = np.zeros((B, Hkv, N, N)); Vp[:, :, np.arange(N), np.arange(N)] = 1.0
+    a = O.attention_with_scores(Q, K, Vp, 0, N, 0, N)
+    p = a["out"].astype(np.float64)                       # [B, N, H, N]: row p's probabilities, bf16-rounded
+    assert np.all(np.triu(p[0, :, 0, :], k=1) == 0.0)      # nothing from the future
+    assert np.allclose(p.sum(axis=3), 1.0, atol=2e-2)
+    assert np.allclose(p[0].sum(axis=0).mean(axis=0), a["score"][0], rtol=2e-2, atol=2e-3)
+
+
 def test_decode_closed_forms():
     r = rng(16)
     B, H, Hkv, cap, D = 2, 4, 2, 12, 8
