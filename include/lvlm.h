@@ -68,7 +68,7 @@ typedef enum {
 
 typedef enum {
     LVLM_OP_SCORE_TOKENS = 0, LVLM_OP_SELECT_TOPK = 1, LVLM_OP_MERGE_COMPACT = 2,
-    LVLM_OP_KV_COMPRESS = 3, LVLM_OP_DECODE_ATTN = 4
+    LVLM_OP_KV_COMPRESS = 3, LVLM_OP_DECODE_ATTN = 4, LVLM_OP_PREFILL_ATTN = 5
 } lvlm_op;
 
 /* Problem sizes.  Each entry point lists the fields it reads; the others are ignored.
@@ -132,6 +132,29 @@ size_t lvlm_workspace_bytes(int op, const lvlm_dims* d);
 lvlm_status lvlm_score_tokens(const void* Q, const void* K, const float* lse,
                               const lvlm_dims* d, float scale,
                               float* score, float* score_head,
+                              void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * The attention of a prefill layer with the importance scores as its by-product (Section 3.2.1, paragraph 3 and
+ * its footnote: the per-key summed scores are what the attention kernel of the layer returns anyway, "to avoid
+ * incurring additional massive computations").  Computes, for every sequence position p and query head h,
+ *     out[b,p,h,:] = softmax_over_visible_keys(Q[b,p,h] . K[b,h/G] * scale) V[b,h/G]
+ *     lse[b,h,p]   = natural log of the sum of the exponentials of row p's scaled logits
+ * and, when `score` is given, exactly what lvlm_score_tokens computes for the window [q_lo, q_hi) of the same
+ * rows - but from the normalisers this attention pass has just produced, so that only the column-sum pass
+ * over the window is paid on top of the attention.
+ *   Q          [B][N][H][D] bf16, row p = sequence position p (strides d->q_stride_*)
+ *   K, V       [B][Hkv][cap][D] bf16, rows 0..N-1 valid (strides d->kv_stride_*)
+ *   out        [B][N][H][D] bf16, packed        lse  [B][H][N] fp32
+ *   score      optional [B][n] fp32; score_head optional [B][Hkv] rows of n fp32, d->head_stride apart
+ *              (needs score); the workspace is only needed with score
+ * Reads d: B,H,Hkv,D,N,cap,causal,q_stride_*,kv_stride_*, and with score also i0,n,q_lo,q_hi,head_stride.
+ * Errors: INVALID_ARG (NULL Q/K/V/out/lse, N>cap, H%Hkv, scale<=0, score_head without score, a bad window),
+ * UNSUPPORTED (D!=128), ALIGNMENT, WORKSPACE.  Contents of the outputs are undefined when a kernel gave up
+ * on a wait and set LVLM_DEV_TIMEOUT (the same holds for lvlm_score_tokens and lvlm_merge_compact).
+ */
+lvlm_status lvlm_prefill_attn(const void* Q, const void* K, const void* V, const lvlm_dims* d, float scale,
+                              void* out, float* lse, float* score, float* score_head,
                               void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
@@ -227,8 +250,9 @@ lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, int32_t* pos,
  * written in the previous decoding step; NOT true right after lvlm_kv_compress or
  * lvlm_merge_compact on the same cache).  The kernel then starts fetching the cache while that
  * operation is still draining; q, k_new, v_new and all writes wait for it as always.
- * Workspace: only used when acc_score is given (the scaled logits are parked there between
- * the pass over the keys and the update of acc_score); its contents need not be zeroed.
+ * Workspace: only used when acc_score is given and the cache is so long that the scaled logits of a CTA's
+ * own keys do not fit in its shared memory (they are then parked there between the pass over the keys and
+ * the update of acc_score); its contents need not be zeroed.
  * Reads d: B,H,Hkv,D,cap,kv_stride_*.
  * Errors: INVALID_ARG, UNSUPPORTED (D!=128, H/Hkv > 8), ALIGNMENT, WORKSPACE.
  */

@@ -19,11 +19,11 @@ _LIB_PATH = os.path.join(_PKG, "liblvlm.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA = range(6)
 DEV_NONFINITE, DEV_TIMEOUT, DEV_BOUNDS = 1, 2, 4
 W_LINEAR_RANK, W_GEOMETRIC, W_UNIFORM, W_CUSTOM, W_NEAREST_KEPT = range(5)
-OP_SCORE_TOKENS, OP_SELECT_TOPK, OP_MERGE_COMPACT, OP_KV_COMPRESS, OP_DECODE_ATTN = range(5)
+OP_SCORE_TOKENS, OP_SELECT_TOPK, OP_MERGE_COMPACT, OP_KV_COMPRESS, OP_DECODE_ATTN, OP_PREFILL_ATTN = range(6)
 
 EXPORTS = ("lvlm_version", "lvlm_status_string", "lvlm_workspace_bytes", "lvlm_score_tokens",
            "lvlm_select_topk", "lvlm_merge_compact", "lvlm_kv_compress", "lvlm_decode_attn",
-           "lvlm_decode_attn_static")
+           "lvlm_decode_attn_static", "lvlm_prefill_attn")
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.lvlm_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, f32, vp, vp, sz, vp, vp]
         L.lvlm_decode_attn_static.restype = ctypes.c_int
         L.lvlm_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, f32, vp, vp, vp]
+        L.lvlm_prefill_attn.restype = ctypes.c_int
+        L.lvlm_prefill_attn.argtypes = [vp, vp, vp, dp, f32, vp, vp, vp, vp, vp, sz, vp, vp]
         _lib = L
     return _lib
 
@@ -159,6 +161,41 @@ def score_tokens(Q, K, *, N, i0, n, q_lo, q_hi, causal=True, scale=None, lse=Non
                                    ctypes.c_float(scale), _ptr(score), _ptr(head), wsp, wsn,
                                    _ptr(dev_status), _stream(stream)), "lvlm_score_tokens")
     return score, head
+
+
+def prefill_attn(Q, K, V, *, N, causal=True, scale=None, window=None, i0=0, n=0, want_head=False,
+                 out=None, lse=None, score_out=None, head_out=None, ws=None, dev_status=None, stream=None):
+    """lvlm_prefill_attn.  Q [B,N,H,D], K, V [B,Hkv,cap,D].  Returns (out [B,N,H,D] bf16, lse [B,H,N],
+    score [B,n] or None, score_head [B,Hkv,n] or None); the scores are asked for with
+    ``window=(q_lo, q_hi)`` and the image span ``i0, n``."""
+    B, Nq, H, D = Q.shape
+    Hkv, cap = K.shape[1], K.shape[2]
+    assert Nq == N and Q.stride(3) == 1 and K.stride(3) == 1 and K.stride(2) == D and V.stride() == K.stride()
+    d = Dims(B=B, H=H, Hkv=Hkv, D=D, N=N, cap=cap, causal=int(causal))
+    d.q_stride_b, d.q_stride_n, d.q_stride_h = Q.stride(0), Q.stride(1), Q.stride(2)
+    d.kv_stride_b, d.kv_stride_h = K.stride(0), K.stride(1)
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    if out is None:
+        out = torch.empty(B, N, H, D, dtype=Q.dtype, device=Q.device)
+    if lse is None:
+        lse = torch.empty(B, H, N, dtype=torch.float32, device=Q.device)
+    score = head = None
+    wsp, wsn = None, 0
+    if window is not None:
+        d.q_lo, d.q_hi, d.i0, d.n = window[0], window[1], i0, n
+        score = score_out if score_out is not None else torch.empty(B, n, dtype=torch.float32, device=Q.device)
+        head = head_out
+        if head is None and want_head:
+            head = torch.empty(B, Hkv, n, dtype=torch.float32, device=Q.device)
+        if head is not None:
+            assert head.stride(2) == 1 and head.stride(0) == Hkv * head.stride(1)
+            d.head_stride = head.stride(1)
+        ws, wsp, wsn = _ws(ws, OP_PREFILL_ATTN, d, Q.device)
+    _check(lib().lvlm_prefill_attn(_ptr(Q), _ptr(K), _ptr(V), ctypes.byref(d), ctypes.c_float(scale), _ptr(out),
+                                   _ptr(lse), _ptr(score), _ptr(head), wsp, wsn, _ptr(dev_status),
+                                   _stream(stream)), "lvlm_prefill_attn")
+    return out, lse, score, head
 
 
 def select_topk(score, k, *, want_kept=True, want_near=False, rank_out=None, kept_out=None,

@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liblvlm.so")
 TEST_LIB = os.path.join(PKG, "liblvlm_test.so")      # the same sources with -DLVLM_TEST_HOOKS, for the tests only
 SOURCES = ["lvlm.cu", "select.cu", "compact.cu", "merge_compact.cu", "kv_compress.cu",
-           "decode.cu", "score.cu", "score_tc.cu", "nearest_kept.cu"]
+           "decode.cu", "score.cu", "score_tc.cu", "nearest_kept.cu", "prefill_attn.cu"]
 
 
 def _nvcc() -> str:

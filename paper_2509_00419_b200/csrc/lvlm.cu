@@ -6,6 +6,7 @@ size_t score_tokens_workspace(const lvlm_dims* d);
 size_t merge_compact_workspace(const lvlm_dims* d);
 size_t kv_compress_workspace(const lvlm_dims* d);
 size_t decode_attn_workspace(const lvlm_dims* d);
+size_t prefill_attn_workspace(const lvlm_dims* d);
 }  // namespace lvlm
 
 // Programmatic dependent launch of the library's kernels is always on in the library proper.  The test build
@@ -45,6 +46,7 @@ extern "C" size_t lvlm_workspace_bytes(int op, const lvlm_dims* d) {
         case LVLM_OP_MERGE_COMPACT: return lvlm::merge_compact_workspace(d);
         case LVLM_OP_KV_COMPRESS: return lvlm::kv_compress_workspace(d);
         case LVLM_OP_DECODE_ATTN: return lvlm::decode_attn_workspace(d);
+        case LVLM_OP_PREFILL_ATTN: return lvlm::prefill_attn_workspace(d);
     }
     return 0;
 }

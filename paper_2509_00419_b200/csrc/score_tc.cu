@@ -382,7 +382,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
 lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, const lvlm_dims* d,
                             const ScoreStrides& st, float scale, float* lse_ws, float* partial,
                             int32_t* cnt, float* score, float* score_head, int32_t* dev_status,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, bool normalisers_ready) {
     const int Nq = d->q_hi - d->q_lo;
     CUtensorMap qmap, kmap;
     {
@@ -420,8 +420,9 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
         }
     }
     a.hsplit = hsplit; a.nkt = nkt; a.ksplit = 1;
-    if (lse) LVLM_RETURN_IF_CUDA(cudaMemsetAsync(cnt, 0, (size_t)d->B * nkt * 4, stream));
-    if (!lse) {
+    const bool skip_pass1 = lse != nullptr || normalisers_ready;
+    if (skip_pass1) LVLM_RETURN_IF_CUDA(cudaMemsetAsync(cnt, 0, (size_t)d->B * nkt * 4, stream));
+    if (!skip_pass1) {
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<0>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         // pass 1: when query tiles x heads do not fill the GPU, a cluster of CTAs shares the key tiles

@@ -479,3 +479,35 @@ def test_results_do_not_depend_on_programmatic_dependent_launch():
     assert not hasattr(L.lib(), "lvlm_debug_set_pdl")        # the library proper exports no switch
     for a, b in zip(plain, overlapped):
         assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ prefill attention with the scores as a by-product
+ATTN_CASES = [  # B, N, H, Hkv, q_lo, i0, n, causal
+    (1, 128, 2, 1, 100, 0, 90, True), (2, 300, 4, 2, 250, 7, 200, True), (1, 517, 7, 1, 400, 3, 390, True),
+    (1, 260, 2, 2, 0, 0, 260, True), (2, 130, 4, 4, 64, 0, 64, False),
+]
+
+
+@pytest.mark.parametrize("case", ATTN_CASES)
+def test_prefill_attn_with_scores(case):
+    B, N, H, Hkv, q_lo, i0, n, causal = case
+    r = np.random.default_rng(N + H)
+    bf = lambda *s: torch.from_numpy(r.normal(size=s).astype(np.float32)).to(torch.bfloat16)
+    Q, K, V = bf(B, N, H, 128), bf(B, Hkv, N + 5, 128), bf(B, Hkv, N + 5, 128)
+    want = O.attention_with_scores(f64(Q), f64(K)[:, :, :N], f64(V)[:, :, :N], q_lo, N, i0, n, causal=causal)
+    flag = status_tensor()
+    out, lse, score, head = L.prefill_attn(Q.cuda(), K.cuda(), V.cuda(), N=N, causal=causal, window=(q_lo, N),
+                                           i0=i0, n=n, want_head=True, dev_status=flag)
+    torch.cuda.synchronize()
+    assert flag.item() == 0
+    assert_rows_close(f64(out), want["out"], what="attention output")
+    assert np.allclose(lse.cpu().numpy(), want["lse"], rtol=1e-3, atol=1e-3)
+    assert_scores_close(f64(score), want["score"], what="score from the attention pass")
+    assert_scores_close(f64(head), want["score_head"], what="score_head from the attention pass")
+    # the same scores as the stand-alone entry point gives (which pays a pass of its own for the normalisers)
+    s2, h2 = L.score_tokens(Q.cuda()[:, q_lo:], K.cuda(), N=N, i0=i0, n=n, q_lo=q_lo, q_hi=N, causal=causal, want_head=True)
+    assert_scores_close(f64(score), f64(s2), what="fused against stand-alone scoring")
+    # attention only: no window, no workspace
+    out2, lse2, none_s, _ = L.prefill_attn(Q.cuda(), K.cuda(), V.cuda(), N=N, causal=causal)
+    torch.cuda.synchronize()
+    assert none_s is None and torch.equal(out2, out) and torch.equal(lse2, lse)
