@@ -172,6 +172,48 @@ def bench_prefill(w, device, steps, warmup, flush, peaks, breakdown=True):
 
 
 # ------------------------------------------------------------------------------------------
+# the layer's attention with the scores as its by-product, against attention + stand-alone scoring
+# ------------------------------------------------------------------------------------------
+def bench_prefill_attn(w, device, steps, warmup, flush, peaks):
+    """Stage-1 layer of ``w``: (a) lvlm_prefill_attn alone plus lvlm_score_tokens on the text window (which pays
+    a pass of its own for the row normalisers), (b) lvlm_prefill_attn asked for the scores itself."""
+    from paper_2509_00419_b200 import binding as L
+    from paper_2509_00419_b200 import inputs as I
+    from paper_2509_00419_b200 import pipeline as P
+    layer = w.stages[0][0]
+    pos = torch.arange(w.N, dtype=torch.int32, device=device)[None].repeat(w.B, 1)
+    q, k, v = I.layer_qkv(w, layer, pos, device)
+    q_lo = w.i0 + w.n
+    out = torch.empty_like(q)
+    lse = torch.empty(w.B, w.H, w.N, dtype=torch.float32, device=device)
+    score = torch.empty(w.B, w.n, dtype=torch.float32, device=device)
+    d = L.Dims(B=w.B, H=w.H, Hkv=w.Hkv, D=128, N=w.N, cap=k.shape[2], i0=w.i0, n=w.n, q_lo=q_lo, q_hi=w.N, causal=1)
+    ws = L.alloc_workspace(L.OP_PREFILL_ATTN, d, device)
+    qwin = q[:, q_lo:]
+
+    def separate():
+        L.prefill_attn(q, k, v, N=w.N, out=out, lse=lse)
+        L.score_tokens(qwin, k, N=w.N, i0=w.i0, n=w.n, q_lo=q_lo, q_hi=w.N, score_out=score, ws=ws)
+
+    def fused():
+        L.prefill_attn(q, k, v, N=w.N, window=(q_lo, w.N), i0=w.i0, n=w.n, out=out, lse=lse, score_out=score, ws=ws)
+
+    def attn_only():
+        L.prefill_attn(q, k, v, N=w.N, out=out, lse=lse)
+
+    t = {}
+    for name, fn in (("attention_only", attn_only), ("attention_then_score_tokens", separate), ("fused", fused)):
+        g = P.capture(fn)
+        t[name], _ = timed(g.replay, steps, warmup, flush)
+        del g
+    flops = 4.0 * w.B * w.H * 128 * (w.N * (w.N + 1) / 2)          # causal: Q K^T and P V
+    return {"ms": t, "attention_tflops": flops / (t["attention_only"] * 1e9),
+            "attention_frac_tensor": flops / (t["attention_only"] * 1e9) / peaks["bf16_tflops"],
+            "scores_cost_ms": {"separate": t["attention_then_score_tokens"] - t["attention_only"],
+                               "fused": t["fused"] - t["attention_only"]}}
+
+
+# ------------------------------------------------------------------------------------------
 # the headline step: prefill pyramid + one-off compression + one decode step
 # ------------------------------------------------------------------------------------------
 class FullPass:
@@ -581,6 +623,11 @@ def summary_table(name, ex):
         row["decode_us_per_layer"] = round(dl["decode_us_per_layer_step"], 2)
         if "compress_frac_hbm" in dl:
             row["kv_compress_hbm"] = round(dl["compress_frac_hbm"], 3)
+    pa = ex.get("prefill_attn")
+    if pa:
+        row["prefill_attn_tensor"] = round(pa["attention_frac_tensor"], 3)
+        row["scores_cost_us_separate_vs_fused"] = [round(pa["scores_cost_ms"]["separate"] * 1e3, 1),
+                                                    round(pa["scores_cost_ms"]["fused"] * 1e3, 1)]
     return row
 
 
@@ -716,6 +763,9 @@ def main():
                     ex["prefill"], run = bench_prefill(wx, device, max(5, args.steps // 2), 3, flush, peaks)
                     del run
                     torch.cuda.empty_cache()
+                    if name in ("cfg3", "cfg5"):
+                        ex["prefill_attn"] = bench_prefill_attn(wx, device, 5, 3, flush, peaks)
+                        torch.cuda.empty_cache()
                 if wx.decode_steps > 1:
                     prompt = wx.N if not wx.stages else wx.stages[-1][1] + wx.T + wx.i0
                     nsteps = args.decode_steps or wx.decode_steps

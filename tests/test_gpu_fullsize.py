@@ -285,3 +285,28 @@ def test_score_all_rows_window(wname, cut):
     # every query row hands out probability 1 over the keys it sees: the per-head sums over ALL keys equal
     # the number of rows, so the image share can never exceed it
     assert float(score.sum(dim=1).max()) <= w.N + 1e-3
+
+
+@pytest.mark.parametrize("wname,cut", [("cfg2", {}), ("cfg5", {"n": 3840, "T": 256})])
+def test_prefill_attn_with_scores_full_size(wname, cut):
+    """The layer's attention with the importance scores as its by-product, at cfg2's size and on a 4096-token
+    cut of cfg5: output, lse and the text-window scores against the oracle; the scores also against the
+    stand-alone entry point."""
+    w = I.shrink(I.WORKLOADS[wname], **cut)
+    dev = torch.device("cuda", 0)
+    layer = w.stages[0][0]
+    pos = torch.arange(w.N, dtype=torch.int32, device=dev)[None].repeat(w.B, 1)
+    q, k, v = I.layer_qkv(w, layer, pos, dev)
+    flag = torch.zeros(1, dtype=torch.int32, device=dev)
+    q_lo = w.i0 + w.n
+    out, lse, score, head = L.prefill_attn(q, k, v, N=w.N, window=(q_lo, w.N), i0=w.i0, n=w.n, want_head=True,
+                                           dev_status=flag)
+    torch.cuda.synchronize()
+    assert int(flag.item()) == 0
+    want = O.attention_with_scores(f64(q), f64(k), f64(v), q_lo, w.N, w.i0, w.n)
+    assert_rows_close(f64(out), want["out"], what=f"{wname} attention output")
+    assert np.allclose(lse.cpu().numpy(), want["lse"], rtol=1e-3, atol=1e-3)
+    assert_scores_close(f64(score), want["score"], what=f"{wname} score from the attention pass")
+    assert_scores_close(f64(head), want["score_head"], what=f"{wname} score_head from the attention pass")
+    s2, _ = L.score_tokens(q[:, q_lo:], k, N=w.N, i0=w.i0, n=w.n, q_lo=q_lo, q_hi=w.N, want_head=False)
+    assert_scores_close(f64(score), f64(s2), what="fused against stand-alone scoring")
