@@ -172,6 +172,30 @@ def bench_prefill(w, device, steps, warmup, flush, peaks, breakdown=True):
 
 
 # ------------------------------------------------------------------------------------------
+# selection on scores that pile up in a few values
+# ------------------------------------------------------------------------------------------
+def bench_select_ties(device):
+    """lvlm_select_topk on one sequence of n scores: spread out, all equal, four distinct values (us, best of 8)."""
+    from paper_2509_00419_b200 import binding as L
+    from paper_2509_00419_b200 import pipeline as P
+    res = {}
+    for n in (16384, 65536):
+        g = torch.Generator().manual_seed(n)
+        cases = {"spread": torch.rand(1, n, generator=g) ** 4, "all_equal": torch.full((1, n), 0.25),
+                 "four_values": torch.randint(0, 4, (1, n), generator=g).float() * 0.125}
+        row = {}
+        for name, sc in cases.items():
+            sc = sc.to(device)
+            rank = torch.empty(1, n, dtype=torch.int32, device=device)
+            gr = P.capture(lambda: L.select_topk(sc, n // 4, want_kept=False, rank_out=rank))
+            ts, _ = timed(gr.replay, 8, 3, None)
+            row[name] = round(ts * 1e3, 1)
+            del gr
+        res[str(n)] = row
+    return res
+
+
+# ------------------------------------------------------------------------------------------
 # the layer's attention with the scores as its by-product, against attention + stand-alone scoring
 # ------------------------------------------------------------------------------------------
 def bench_prefill_attn(w, device, steps, warmup, flush, peaks):
@@ -838,6 +862,7 @@ def main():
                                 "mean_kept_fraction": float((kept / img_before).mean().item())}
         fp.restore()
         extras["beta_sweep_" + w.name] = sweep
+        extras["select_ties_us"] = bench_select_ties(device)
         out["workloads"] = extras
     elif rank == 0:
         out["e2e"] = {"value": None, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,

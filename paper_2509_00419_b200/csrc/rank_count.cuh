@@ -3,9 +3,11 @@
 // nearest-kept merge.  A CTA holds one slice of the keys in shared memory and every thread counts
 // for its own key; the CTAs of a cluster (one per slice, along y) add their counts through
 // distributed shared memory.  A short slice is simply read through.  A long slice is first put into
-// 1024 bins by the high word of the key (linear between the slice's smallest and largest high word):
-// all keys of lower bins are smaller, so only the thread's own bin is read through.  How the keys
-// happen to be ordered inside a bin does not matter, the count is the same.
+// 1024 bins - linear in the high word of the key, or, where that leaves a bin deeper than 256 keys (ties, a
+// handful of distinct scores), bounded by a sorted sample of the slice's own keys: the keys are distinct
+// (the index is their low word), so such bins stay a few keys deep whatever the scores look like.  All
+// keys of lower bins are smaller, so only the thread's own bin is read through; how the keys happen to
+// be ordered inside a bin does not matter, the count is the same.
 #pragma once
 #include "common.cuh"
 
@@ -21,7 +23,8 @@ constexpr int kRankMaxJT = 4;              // keys a thread ranks when the slice
 
 // Shared memory a CTA needs for a slice of slice_len keys.
 inline size_t rank_smem_bytes(int slice_len) {
-    return slice_len >= kRankBinFrom ? (size_t)slice_len * 16 + (size_t)(2 * kRankBins + 2) * 4 : (size_t)slice_len * 8;
+    return slice_len >= kRankBinFrom ? (size_t)slice_len * 16 + (size_t)kRankBins * 8 + (size_t)(2 * kRankBins + 2) * 4
+                                     : (size_t)slice_len * 8;
 }
 
 __device__ __forceinline__ uint32_t rank_cluster_rank() {
@@ -39,6 +42,22 @@ __device__ __forceinline__ int rank_ld_cluster(const int* my_smem, uint32_t rank
     int v;
     asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
     return v;
+}
+
+// Ascending sort of P (a power of two) 64-bit keys in shared memory by the whole CTA.
+__device__ __forceinline__ void rank_bitonic_sort(uint64_t* keys, int P) {
+    for (int k2 = 2; k2 <= P; k2 <<= 1) {
+        for (int j = k2 >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < (P >> 1); t += blockDim.x) {
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const int l = i | j;
+                const bool up = (i & k2) == 0;
+                const uint64_t a = keys[i], b = keys[l];
+                if ((a > b) == up) { keys[i] = b; keys[l] = a; }
+            }
+            __syncthreads();
+        }
+    }
 }
 
 // Number of slices (cluster size) and keys per slice for n keys in each of B sequences: up to eight
@@ -78,13 +97,15 @@ __device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int
     }
     __syncthreads();
     if (slice_len >= kRankBinFrom) {
-        __shared__ uint32_t s_min[kRankThreads / 32], s_max[kRankThreads / 32];
         __shared__ int s_scan[33];
+        __shared__ uint32_t s_min[kRankThreads / 32], s_max[kRankThreads / 32];
+        __shared__ int s_deepest;
         uint64_t* sb = sk + slice_len;                                   // the keys again, bin by bin
-        int* start = reinterpret_cast<int*>(sb + slice_len);             // [kRankBins + 1]
+        uint64_t* spl = sb + slice_len;                                  // [kRankBins] sorted sample: bin boundaries
+        int* start = reinterpret_cast<int*>(spl + kRankBins);            // [kRankBins + 1]
         int* cursor = start + kRankBins + 1;                             // [kRankBins]
         const int nvalid = max(0, min(slice_len, n - i_lo));
-        // smallest and largest high word of the slice
+        // First try: bins linear in the high word between the slice's extremes (one multiply per key).
         uint32_t lo = 0xFFFFFFFFu, hi = 0u;
         for (int i = tid; i < nvalid; i += kRankThreads) {
             const uint32_t h = (uint32_t)(sk[i] >> 32);
@@ -96,14 +117,50 @@ __device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int
             hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
         }
         if ((tid & 31) == 0) { s_min[tid >> 5] = lo; s_max[tid >> 5] = hi; }
+        if (tid == 0) s_deepest = 0;
         for (int i = tid; i <= kRankBins; i += kRankThreads) start[i] = 0;
         __syncthreads();
 #pragma unroll
         for (int wv = 0; wv < kRankThreads / 32; ++wv) { lo = min(lo, s_min[wv]); hi = max(hi, s_max[wv]); }
         const uint64_t span = (uint64_t)(hi - lo) + 1;                   // hi >= lo whenever the slice has keys
-        auto bin_of = [&](uint32_t h) { return (int)(((uint64_t)(h - lo) * kRankBins) / span); };
-        for (int i = tid; i < nvalid; i += kRankThreads) atomicAdd(&start[bin_of((uint32_t)(sk[i] >> 32))], 1);
+        auto bin_linear = [&](uint64_t key) {
+            const uint32_t h = (uint32_t)(key >> 32);
+            if (h <= lo) return 0;
+            if (h >= hi) return kRankBins - 1;
+            return (int)(((uint64_t)(h - lo) * kRankBins) / span);
+        };
+        // bin of a key = number of boundaries spl[1..1023] that are <= key (binary search), 0 .. 1023
+        auto bin_sampled = [&](uint64_t key) {
+            int lo_i = 0, hi_i = kRankBins - 1;                          // boundaries spl[1 + lo_i .. 1 + hi_i)
+            while (lo_i < hi_i) {
+                const int mid = (lo_i + hi_i) >> 1;
+                if (spl[1 + mid] <= key) lo_i = mid + 1; else hi_i = mid;
+            }
+            return lo_i;
+        };
+        for (int i = tid; i < nvalid; i += kRankThreads) {
+            const int c = atomicAdd(&start[bin_linear(sk[i])], 1) + 1;
+            if (c > 256) atomicMax(&s_deepest, c);                       // (rarely taken)
+        }
         __syncthreads();
+        // Scores that pile up in a few values (ties, a handful of distinct numbers) would make a bin as deep as the
+        // slice.  Then the bins are rebuilt with boundaries taken from a sorted sample of the slice's own keys:
+        // the keys are distinct (the index is their low word), so those bins are a few keys deep whatever
+        // the scores look like.
+        const bool sampled = s_deepest > 256;
+        __syncthreads();
+        if (sampled) {
+            for (int t = tid; t < kRankBins; t += kRankThreads) {
+                const int i = nvalid >= kRankBins ? (int)(((int64_t)t * nvalid) / kRankBins) : t;
+                spl[t] = i < nvalid ? sk[i] : ~0ull;                     // padding sorts last and bounds nothing
+            }
+            for (int i = tid; i <= kRankBins; i += kRankThreads) start[i] = 0;
+            __syncthreads();
+            rank_bitonic_sort(spl, kRankBins);
+            for (int i = tid; i < nvalid; i += kRankThreads) atomicAdd(&start[bin_sampled(sk[i])], 1);
+            __syncthreads();
+        }
+        auto bin_of = [&](uint64_t key) { return sampled ? bin_sampled(key) : bin_linear(key); };
         {   // exclusive scan of the bin counts: four bins per thread
             int c4[4], sum = 0;
 #pragma unroll
@@ -117,21 +174,17 @@ __device__ __forceinline__ bool rank_by_counting(KeyFn key_of, int n, int S, int
         __syncthreads();
         for (int i = tid; i < nvalid; i += kRankThreads) {
             const uint64_t key = sk[i];
-            sb[atomicAdd(&cursor[bin_of((uint32_t)(key >> 32))], 1)] = key;
+            sb[atomicAdd(&cursor[bin_of(key)], 1)] = key;
         }
         __syncthreads();
 #pragma unroll
         for (int u = 0; u < kRankMaxJT; ++u) {
             const uint64_t kj = kjs[u];
-            const uint32_t hj = (uint32_t)(kj >> 32);
             int cnt = 0;
             if (nvalid > 0 && u < jt && rank_key_index(jt, u) < n) {
-                if (hj > hi) cnt = nvalid;
-                else if (hj >= lo) {
-                    const int bj = bin_of(hj);
-                    cnt = start[bj];
-                    for (int p = start[bj]; p < start[bj + 1]; ++p) cnt += sb[p] < kj;
-                }
+                const int bj = bin_of(kj);
+                cnt = start[bj];
+                for (int p = start[bj]; p < start[bj + 1]; ++p) cnt += sb[p] < kj;
             }
             count[u] = cnt;
         }
