@@ -347,6 +347,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     // every copy issued has landed: the compute warps have waited for each stage; the ring is free
     __syncthreads();
     if (s_abort) {                             // a wait gave up: copies may still be in flight, let them land
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         __syncthreads();
     }

@@ -573,6 +573,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) row_stream_kernel(const Str
     }
     __syncthreads();
     if (s_abort) {                                             // copies may still be in flight: let them land
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         __syncthreads();
     }

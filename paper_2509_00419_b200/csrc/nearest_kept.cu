@@ -523,6 +523,7 @@ nk_sim_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (sm->abort) {
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
     if (warp == 1) {

@@ -308,6 +308,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
     tc_fence_before();
     __syncthreads();
     if (sm->abort) {                              // let copies still in flight land before leaving
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
     if (warp == 1) {

@@ -49,7 +49,7 @@ struct TcSmem {
     uint32_t tmem_base;
     volatile int abort;
     volatile int last;
-    float lse_s[8][2][kTile / 2];  // per epilogue warp, per accumulator buffer: normalisers of its 64 columns
+    alignas(16) float lse_s[8][2][kTile / 2];  // per epilogue warp, per accumulator buffer: normalisers of its 64 columns
     float xm[kTile], xl[kTile];    // what the warps of the upper column half hand to the lower half
 };
 
@@ -113,10 +113,12 @@ __device__ __forceinline__ void rowstat_chunk(float* v, int lim, float scale_log
 __device__ __forceinline__ float colsum_chunk(const float* v, const float* ls, int first, float scale_log2) {
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
     if (first <= 0) {
+        const float4* ls4 = reinterpret_cast<const float4*>(ls);         // 16-byte aligned: four normalisers a load
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
-            s0 += ex2_fast(fmaf(v[c], scale_log2, -ls[c])); s1 += ex2_fast(fmaf(v[c + 1], scale_log2, -ls[c + 1]));
-            s2 += ex2_fast(fmaf(v[c + 2], scale_log2, -ls[c + 2])); s3 += ex2_fast(fmaf(v[c + 3], scale_log2, -ls[c + 3]));
+            const float4 l = ls4[c >> 2];
+            s0 += ex2_fast(fmaf(v[c], scale_log2, -l.x)); s1 += ex2_fast(fmaf(v[c + 1], scale_log2, -l.y));
+            s2 += ex2_fast(fmaf(v[c + 2], scale_log2, -l.z)); s3 += ex2_fast(fmaf(v[c + 3], scale_log2, -l.w));
         }
     } else {
 #pragma unroll
@@ -371,6 +373,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
         cluster_barrier_all();
     }
     if (sm->abort) {                              // let copies still in flight land before leaving
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
     if (warp == 1) {
@@ -426,9 +429,18 @@ lvlm_status launch_score_tc(const void* Q, const void* K, const float* lse, cons
         LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(score_tc_kernel<0>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         // pass 1: when query tiles x heads do not fill the GPU, a cluster of CTAs shares the key tiles
+        // (the split with the smallest estimate waves x (fixed + key tiles per CTA x per-tile), as for pass 2)
         int ksplit = 1;
         const int max_kt = (d->N + kTile - 1) / kTile;
-        while (ksplit < 8 && (int64_t)nqt * d->H * d->B * ksplit < 148 && 2 * ksplit <= max_kt) ksplit *= 2;
+        {
+            double best = 1e30;
+            for (int ks = 1; ks <= 8 && ks <= max_kt; ++ks) {
+                const int64_t ctas = (int64_t)nqt * d->H * d->B * ks;
+                const double waves = (double)((ctas + 295) / 296);
+                const double est = waves * (5.0 + 0.6 * ((max_kt + ks - 1) / ks));
+                if (est < best - 1e-9) { best = est; ksplit = ks; }
+            }
+        }
         a.ksplit = ksplit;
         const lvlm_status s0 = launch_kernel(score_tc_kernel<0>, dim3(nqt * ksplit, d->H, d->B), dim3(kTcThreads),
                                              smem, stream, ksplit, qmap, kmap, a);

@@ -38,6 +38,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
 // so that waiting warps leave the issue slots to the warps that work.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_u32(bar);
+#pragma unroll 1
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         uint32_t done;
         asm volatile(
