@@ -440,6 +440,7 @@ def bench_decode_loop(w, device, flush, peaks, prompt_len, steps_total):
                 first_drop = (~kept).float().argmax(dim=-1)
                 moved_rows_first = int((w.budget - first_drop).clamp(min=0).sum().item())
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            flush()                       # keeps the GPU busy while the replay is enqueued: the events then bracket device time
             e0.record(); g_cmp.replay(); e1.record()
             evs.append(("c", e0, e1))
             cur_len, n_cmp = w.budget, n_cmp + 1

@@ -32,7 +32,7 @@ size_t kv_compress_workspace(const lvlm_dims* d) {
 // Score in integer units of 2^-24 (negative and non-finite scores count as zero).
 __device__ __forceinline__ long long score_units(float s) {
     if (!(s > 0.f) || (__float_as_uint(s) & 0x7F800000u) == 0x7F800000u) return 0;
-    return __float2ll_rn(ldexpf(s, 24));
+    return __float2ll_rn(s * 16777216.0f);               // exact: a power of two (beyond 2^104 both saturate)
 }
 
 // ceil(a * b / c) for a, b < 2^63, c = 10^6, in 128-bit arithmetic.
@@ -43,6 +43,7 @@ __device__ __forceinline__ unsigned long long ceil_muldiv(unsigned long long a, 
     // assumed: reduce hi first.
     unsigned long long rem = hi % c;
     unsigned long long q = 0;
+#pragma unroll 1
     for (int bit = 63; bit >= 0; --bit) {
         rem = (rem << 1) | ((lo >> bit) & 1ull);        // rem < 2c < 2^63, no overflow
         q <<= 1;
@@ -251,9 +252,19 @@ kv_plan_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __re
     }
 }
 
-// The same for caches of up to 2048 rows: one WARP per (sequence, KV head), a lane holds KPL consecutive
-// entries, every sum is a handful of shuffles and no barrier is needed, so an SM works on dozens of heads at once.
-template <int KPL>
+// The same for caches of up to 2048 rows: one WARP per (sequence, KV head); lane l holds entries l, l + 32, ...
+// (coalesced), every sum is a handful of shuffles and no barrier is needed, so an SM works on dozens of heads at
+// once.  Only the 32-bit image of the score is searched: among entries of equal score the lower index comes first,
+// so once the threshold score T is known, "the first `need` entries of score T" is a running count in index order
+// and the index never has to enter the key.  The searches are loops over registers; the pass that writes the map
+// is a loop over the entries that reads the scores again (they are in L1), which keeps the kernel's code short:
+// a warp runs through it once, and straight-line code is fetched slower than it executes.
+// MASS: the threshold beta is in use (without it only the budget's count search is compiled in).
+__device__ __forceinline__ void plan_cp_async4(void* smem, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+
+template <int KPL, bool MASS>
 __global__ void __launch_bounds__(128)
 kv_plan_warp_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t* __restrict__ e_lo,
                     const int32_t* __restrict__ e_hi, int heads, int Hkv, int cap, int recent, int only_small,
@@ -283,124 +294,151 @@ kv_plan_warp_kernel(float* acc_score, int32_t* pos, int32_t* len, const int32_t*
     const int m = hi - lo;
     if (only_small && m > 32 * KPL) return;              // too many entries for the registers: the CTA kernel plans it
 
-    const int j0 = lane * KPL;
-    uint64_t key[KPL];
-    constexpr bool kKeepUnits = KPL <= 32;               // the scores in integer units stay in registers when they fit
-    unsigned long long un[kKeepUnits ? KPL : 1];
+    // The scores and the position ids of the evictable entries come to shared memory by asynchronous copies
+    // (all of them in flight at once); the scores are turned into keys there, by a loop over the entries, and
+    // then taken into registers.
+    extern __shared__ __align__(16) uint32_t s_plan[];   // per warp: [KPL * 32] keys, [KPL * 32] position ids
+    uint32_t* my_hk = s_plan + (threadIdx.x >> 5) * (2 * KPL * 32);
+    uint32_t* my_pos = my_hk + KPL * 32;
+    const int32_t* ps = pos ? pos + (int64_t)m_idx * cap : nullptr;
+#pragma unroll 4
+    for (int j = lane; j < m; j += 32) {
+        plan_cp_async4(&my_hk[j], acc + lo + j);
+        if (ps) plan_cp_async4(&my_pos[j], ps + lo + j);
+    }
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+    __syncwarp();
+    uint32_t k_and = ~0u, k_or = 0u;
     bool nonfinite = false;
-    uint64_t k_and = ~0ull, k_or = 0ull;
-    unsigned long long total = 0;
-#pragma unroll
-    for (int u = 0; u < KPL; ++u) {
-        key[u] = ~0ull;                                  // past the end: above every real key
-        if (kKeepUnits) un[u] = 0ull;
-        if (j0 + u < m) {
-            const float sv = acc[lo + j0 + u];
-            key[u] = ((uint64_t)desc_key(sv, &nonfinite) << 32) | (uint32_t)(j0 + u);
-            k_and &= key[u]; k_or |= key[u];
-            const unsigned long long su = (unsigned long long)score_units(sv);
-            if (kKeepUnits) un[u] = su;
-            total += su;
-        }
+#pragma unroll 4
+    for (int j = lane; j < KPL * 32; j += 32) {
+        uint32_t h = ~0u;                                // past the end: the top value
+        if (j < m) { h = desc_key(__uint_as_float(my_hk[j]), &nonfinite); k_and &= h; k_or |= h; }
+        my_hk[j] = h;
     }
     if (nonfinite && dev_status) atomicOr(dev_status, LVLM_DEV_NONFINITE);
+    uint32_t hk[KPL];                                    // ascending = descending score
+#pragma unroll
+    for (int u = 0; u < KPL; ++u) hk[u] = my_hk[u * 32 + lane];       // (written by this very lane)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         k_and &= __shfl_xor_sync(0xFFFFFFFFu, k_and, o);
         k_or |= __shfl_xor_sync(0xFFFFFFFFu, k_or, o);
-        total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
     }
-    const uint64_t diff = m > 0 ? (k_and ^ k_or) : 0ull;
-    auto units_of = [](uint64_t k) -> unsigned long long {
-        const uint32_t dk = (uint32_t)(k >> 32);
+    const uint32_t diff = m > 0 ? (k_and ^ k_or) : 0u;
+    auto units_of = [](uint32_t dk) -> unsigned long long {      // the score units behind a key
         if (dk == 0xFFFFFFFFu) return 0ull;
         const uint32_t asc = ~dk;
         const uint32_t bits = (asc & 0x80000000u) ? (asc & 0x7FFFFFFFu) : ~asc;
         return (unsigned long long)score_units(__uint_as_float(bits));
     };
-    auto search_count = [&](int target) -> uint64_t {
-        uint64_t ans = k_and, todo = diff;
-        while (todo) {
-            const int bit = 63 - __clzll((long long)todo);
-            todo &= ~(1ull << bit);
-            const uint64_t cand = (ans & ~(1ull << bit)) | ((1ull << bit) - 1ull);
-            int cnt = 0;
+    // Score units of the entries with key <= cand (or < cand), summed over the warp.
+    auto mass_upto = [&](uint32_t cand, bool strict) -> unsigned long long {
+        unsigned long long ms = 0;
 #pragma unroll
-            for (int u = 0; u < KPL; ++u) cnt += key[u] <= cand;
-            cnt = warp_sum(cnt);
-            if (cnt >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
+        for (int u = 0; u < KPL; ++u) {
+            uint32_t h = hk[u];
+            if (KPL > 32) asm volatile("" : "+r"(h));    // worked out again at every use: 64 more registers would not fit
+            if (strict ? h < cand : h <= cand) ms += units_of(h);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ms += __shfl_xor_sync(0xFFFFFFFFu, ms, o);
+        return ms;
+    };
+    // Smallest score key T such that the entries with key <= T are at least `target` many (by_count) or hold at
+    // least `target` units of score: built bit by bit from the top, over the bits in which the keys differ.
+    // Entries past the end carry the top key and no score: they are counted only where every real entry is.
+    auto search = [&](unsigned long long target, bool by_count) -> uint32_t {
+        uint32_t ans = k_and, todo = diff;
+#pragma unroll 1
+        while (todo) {
+            const int bit = 31 - __clz((int)todo);
+            todo &= ~(1u << bit);
+            const uint32_t cand = (ans & ~(1u << bit)) | ((1u << bit) - 1u);
+            unsigned long long have;
+            if (!MASS || by_count) {
+                int cnt = 0;
+#pragma unroll
+                for (int u = 0; u < KPL; ++u) cnt += hk[u] <= cand;
+                have = (unsigned long long)warp_sum(cnt);
+            } else {
+                have = mass_upto(cand, false);
+            }
+            if (have >= target) ans &= ~(1u << bit); else ans |= 1u << bit;
         }
         return ans;
     };
-    auto search_mass = [&](unsigned long long target) -> uint64_t {
-        uint64_t ans = k_and, todo = diff;
-        while (todo) {
-            const int bit = 63 - __clzll((long long)todo);
-            todo &= ~(1ull << bit);
-            const uint64_t cand = (ans & ~(1ull << bit)) | ((1ull << bit) - 1ull);
-            unsigned long long ms = 0;
+    auto count_below = [&](uint32_t T) -> int {          // entries with a strictly better score than T
+        int c = 0;
 #pragma unroll
-            for (int u = 0; u < KPL; ++u) if (key[u] <= cand) ms += kKeepUnits ? un[u] : units_of(key[u]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) ms += __shfl_xor_sync(0xFFFFFFFFu, ms, o);
-            if (ms >= target) ans &= ~(1ull << bit); else ans |= 1ull << bit;
-        }
-        return ans;
+        for (int u = 0; u < KPL; ++u) c += hk[u] < T;
+        return warp_sum(c);
     };
 
+    // ---- how many entries reach the threshold, how many the budget allows --------------------------------------
     int k_beta = m;
-    uint64_t T = ~0ull;                                  // keys <= T survive
+    uint32_t T = ~0u;                                    // survivors: score key < T, and the first `need` entries of key T
+    int need = 0;
     bool have_T = false;
-    if (beta_ppm < 1000000ull && m > 0) {
+    if (MASS && m > 0) {
+        const unsigned long long total = mass_upto(~0u, false);
         const unsigned long long thr = ceil_muldiv(beta_ppm, total, 1000000ull);
         if (thr == 0) k_beta = 1;
         else {
-            T = search_mass(thr);
-            int cnt = 0;
-#pragma unroll
-            for (int u = 0; u < KPL; ++u) cnt += key[u] <= T;
-            k_beta = warp_sum(cnt);
+            T = search(thr, false);
+            const int c = count_below(T);
+            const unsigned long long below = mass_upto(T, true);
+            const unsigned long long each = units_of(T);                 // > 0: the entries of key T are needed
+            need = (int)((thr - below + each - 1ull) / each);
+            k_beta = c + need;
             have_T = true;
         }
     }
     int kc = k_beta;
     if (budget > 0) kc = min(kc, budget - (ln - m));
     kc = min(max(kc, 0), m);
-    if (kc < m && kc > 0 && !(have_T && kc == k_beta)) T = search_count(kc);
+    if (kc < m && kc > 0 && !(have_T && kc == k_beta)) {
+        T = search((unsigned long long)kc, true);
+        need = kc - count_below(T);
+    }
 
-    // survivor map: my entries are consecutive, so a scan of the counts over the lanes gives their places
-    int cnt = 0, first_drop = m;
-#pragma unroll
-    for (int u = 0; u < KPL; ++u) {
-        if (j0 + u < m) {
-            const bool kept = kc >= m || (kc > 0 && key[u] <= T);
-            if (kept) ++cnt; else if (first_drop == m) first_drop = j0 + u;
-        }
-    }
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    int off = incl - cnt;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) first_drop = min(first_drop, __shfl_xor_sync(0xFFFFFFFFu, first_drop, o));
+    // ---- the survivor map, in index order: 32 entries a round, places by ballot ---------------------------------
     float* an = acc_new + (int64_t)m_idx * cap;
-    const int32_t* ps = pos ? pos + (int64_t)m_idx * cap : nullptr;
     int32_t* pn = pos_new + (int64_t)m_idx * cap;
-#pragma unroll
-    for (int u = 0; u < KPL; ++u)
-        if (j0 + u < m && (kc >= m || (kc > 0 && key[u] <= T))) {
-            src[lo + off] = lo + j0 + u;
-            an[lo + off] = acc[lo + j0 + u];
-            if (ps) pn[lo + off] = ps[lo + j0 + u];
-            ++off;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int first_drop = m;
+    if (kc < m) {
+        int base = 0, eq_base = 0;
+#pragma unroll 2
+        for (int j0 = 0; j0 < m; j0 += 32) {
+            const int j = j0 + lane;
+            const bool valid = j < m;
+            const float sv = valid ? acc[lo + j] : 0.f;
+            bool nf = false;
+            const uint32_t h = valid ? desc_key(sv, &nf) : ~0u;
+            const bool is_eq = valid && h == T;
+            const uint32_t beq = __ballot_sync(0xFFFFFFFFu, is_eq);
+            const bool kept = valid && kc > 0 && (h < T || (is_eq && eq_base + __popc(beq & lt_mask) < need));
+            const uint32_t bk = __ballot_sync(0xFFFFFFFFu, kept);
+            if (kept) {
+                const int o = lo + base + __popc(bk & lt_mask);
+                src[o] = lo + j;
+                an[o] = sv;
+                if (ps) pn[o] = (int32_t)my_pos[j];
+            }
+            const uint32_t bd = __ballot_sync(0xFFFFFFFFu, valid && !kept);
+            if (first_drop == m && bd) first_drop = j0 + __ffs((int)bd) - 1;
+            base += __popc(bk);
+            eq_base += __popc(beq);
         }
+    }
     const int new_len = lo + kc + (ln - hi);
+    // rows that do not move (everything when nothing is evicted) and the rows behind the evictable range
     for (int o = lane; o < new_len; o += 32) {
-        if (o < lo) src[o] = o;
-        else if (o >= lo + kc) {
+        if (o < lo || kc >= m) {
+            src[o] = o;
+            if (o >= lo) { an[o] = acc[o]; if (ps) pn[o] = ps[o]; }
+        } else if (o >= lo + kc) {
             const int sidx = hi + (o - lo - kc);
             src[o] = sidx;
             an[o] = acc[sidx];
@@ -441,26 +479,28 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
     const unsigned long long beta_ppm = (unsigned long long)llrint((double)beta * 1.0e6);
     const int heads = d->B * d->Hkv;
     lvlm_status st;
-#define LVLM_PLAN_WARP(KPL_, SMALL_)                                                                             \
-    st = launch_kernel(kv_plan_warp_kernel<KPL_>, dim3((heads + 3) / 4), dim3(128), 0, stream, 1, acc_score, pos, len, \
-                       e_lo, e_hi, heads, d->Hkv, d->cap, d->recent, SMALL_, beta_ppm, budget, src_map, meta, nout,   \
-                       acc_new, pos_new, dev_status)
-    const bool many = heads >= 4 * 148;                 // enough heads to fill the GPU with one warp each
+#define LVLM_PLAN_WARP_(KPL_, SMALL_, MASS_)                                                                     \
+    (cudaFuncSetAttribute(kv_plan_warp_kernel<KPL_, MASS_>, cudaFuncAttributeMaxDynamicSharedMemorySize,              \
+                          4 * 2 * KPL_ * 32 * 4) != cudaSuccess                                                       \
+         ? LVLM_ERR_CUDA                                                                                             \
+         : launch_kernel(kv_plan_warp_kernel<KPL_, MASS_>, dim3((heads + 3) / 4), dim3(128), 4 * 2 * KPL_ * 32 * 4,   \
+                         stream, 1, acc_score, pos, len, e_lo, e_hi, heads, d->Hkv, d->cap, d->recent, SMALL_,        \
+                         beta_ppm, budget, src_map, meta, nout, acc_new, pos_new, dev_status))
+#define LVLM_PLAN_WARP(KPL_, SMALL_) \
+    st = beta_ppm < 1000000ull ? LVLM_PLAN_WARP_(KPL_, SMALL_, true) : LVLM_PLAN_WARP_(KPL_, SMALL_, false)
+    // A warp per head wherever a head's entries fit a warp's registers (no barrier in the searches); a CTA per head
+    // for the others.
     const int kpt = d->cap <= 4096 ? 4 : 16;
     int threads = ((d->cap + kpt - 1) / kpt + 31) / 32 * 32;
     threads = threads < 64 ? 64 : threads;
-    int min_m = 0;                                       // heads the CTA kernel leaves to the warp kernel
-    bool cta_kernel = true;
-    if (many) {
-        if (d->cap <= 512) LVLM_PLAN_WARP(16, 0);
-        else if (d->cap <= 1024) LVLM_PLAN_WARP(32, 0);
-        else if (d->cap <= 1536) LVLM_PLAN_WARP(48, 0);
-        else if (d->cap <= 2048) LVLM_PLAN_WARP(64, 0);
-        else LVLM_PLAN_WARP(32, 1);                      // long caches: the heads with up to 1024 evictable entries
-        if (st != LVLM_OK) return st;
-        cta_kernel = d->cap > 2048;                      // ... the others get a CTA each
-        min_m = 32 * 32 + 1;
-    }
+    if (d->cap <= 512) LVLM_PLAN_WARP(16, 0);
+    else if (d->cap <= 1024) LVLM_PLAN_WARP(32, 0);
+    else if (d->cap <= 1536) LVLM_PLAN_WARP(48, 0);
+    else if (d->cap <= 2048) LVLM_PLAN_WARP(64, 0);
+    else LVLM_PLAN_WARP(32, 1);                          // long caches: the heads with up to 1024 evictable entries
+    if (st != LVLM_OK) return st;
+    const bool cta_kernel = d->cap > 2048;               // ... the others get a CTA each
+    const int min_m = 32 * 32 + 1;                       // heads the CTA kernel leaves to the warp kernel
     if (cta_kernel) {
         // a CTA per head, a thread holds 4 entries (caches up to 4096 rows) or 16; warps without entries leave at once
         st = kpt == 4 ? launch_kernel(kv_plan_kernel<4>, dim3(d->Hkv, d->B), dim3(threads), 0, stream, 1, acc_score, pos,
@@ -471,6 +511,7 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
                                       meta, nout, acc_new, pos_new, dev_status);
     }
 #undef LVLM_PLAN_WARP
+#undef LVLM_PLAN_WARP_
     if (st != LVLM_OK) return st;
     CompactJob j;
     j.base0 = Kc; j.base1 = Vc; j.stride_b = kv_sb * 2; j.stride_g = kv_sh * 2; j.B = d->B; j.G = d->Hkv;

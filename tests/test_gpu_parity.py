@@ -192,6 +192,8 @@ KV_CASES = [  # B, Hkv, cap, beta, budget, recent, use_range
     (2, 3, 64, 0.995, 0, 0, True), (2, 2, 200, 0.9, 0, 0, False), (1, 8, 1024, 1.0, 256, 0, False),
     (3, 2, 1152, 1.0, 1024, 128, False), (2, 4, 333, 0.5, 100, 16, True), (1, 1, 5, 0.7, 0, 0, False),
     (1, 2, 8192, 0.99, 0, 0, True), (1, 2, 9000, 0.97, 4000, 64, False), (2, 2, 2048, 0.995, 0, 0, False),
+    (1, 2, 3000, 0.99, 0, 0, False), (2, 2, 4096, 1.0, 2500, 32, True), (2, 3, 1536, 0.98, 700, 8, False),
+    (40, 16, 96, 0.9, 40, 4, False),
 ]
 
 
