@@ -488,19 +488,24 @@ extern "C" lvlm_status lvlm_kv_compress(void* Kc, void* Vc, float* acc_score, in
                          beta_ppm, budget, src_map, meta, nout, acc_new, pos_new, dev_status))
 #define LVLM_PLAN_WARP(KPL_, SMALL_) \
     st = beta_ppm < 1000000ull ? LVLM_PLAN_WARP_(KPL_, SMALL_, true) : LVLM_PLAN_WARP_(KPL_, SMALL_, false)
-    // A warp per head wherever a head's entries fit a warp's registers (no barrier in the searches); a CTA per head
-    // for the others.
+    // With enough heads to fill the GPU with one warp each, a warp per head (no barrier in the searches); a CTA per
+    // head otherwise, and for the heads whose entries do not fit a warp's registers.
+    const bool many = heads >= 4 * 148;
     const int kpt = d->cap <= 4096 ? 4 : 16;
     int threads = ((d->cap + kpt - 1) / kpt + 31) / 32 * 32;
     threads = threads < 64 ? 64 : threads;
-    if (d->cap <= 512) LVLM_PLAN_WARP(16, 0);
-    else if (d->cap <= 1024) LVLM_PLAN_WARP(32, 0);
-    else if (d->cap <= 1536) LVLM_PLAN_WARP(48, 0);
-    else if (d->cap <= 2048) LVLM_PLAN_WARP(64, 0);
-    else LVLM_PLAN_WARP(32, 1);                          // long caches: the heads with up to 1024 evictable entries
-    if (st != LVLM_OK) return st;
-    const bool cta_kernel = d->cap > 2048;               // ... the others get a CTA each
-    const int min_m = 32 * 32 + 1;                       // heads the CTA kernel leaves to the warp kernel
+    int min_m = 0;                                       // heads the CTA kernel leaves to the warp kernel
+    bool cta_kernel = true;
+    if (many) {
+        if (d->cap <= 512) LVLM_PLAN_WARP(16, 0);
+        else if (d->cap <= 1024) LVLM_PLAN_WARP(32, 0);
+        else if (d->cap <= 1536) LVLM_PLAN_WARP(48, 0);
+        else if (d->cap <= 2048) LVLM_PLAN_WARP(64, 0);
+        else LVLM_PLAN_WARP(32, 1);                      // long caches: the heads with up to 1024 evictable entries
+        if (st != LVLM_OK) return st;
+        cta_kernel = d->cap > 2048;                      // ... the others get a CTA each
+        min_m = 32 * 32 + 1;
+    }
     if (cta_kernel) {
         // a CTA per head, a thread holds 4 entries (caches up to 4096 rows) or 16; warps without entries leave at once
         st = kpt == 4 ? launch_kernel(kv_plan_kernel<4>, dim3(d->Hkv, d->B), dim3(threads), 0, stream, 1, acc_score, pos,

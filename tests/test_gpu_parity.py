@@ -193,7 +193,8 @@ KV_CASES = [  # B, Hkv, cap, beta, budget, recent, use_range
     (3, 2, 1152, 1.0, 1024, 128, False), (2, 4, 333, 0.5, 100, 16, True), (1, 1, 5, 0.7, 0, 0, False),
     (1, 2, 8192, 0.99, 0, 0, True), (1, 2, 9000, 0.97, 4000, 64, False), (2, 2, 2048, 0.995, 0, 0, False),
     (1, 2, 3000, 0.99, 0, 0, False), (2, 2, 4096, 1.0, 2500, 32, True), (2, 3, 1536, 0.98, 700, 8, False),
-    (40, 16, 96, 0.9, 40, 4, False),
+    (40, 16, 96, 0.9, 40, 4, False), (37, 16, 1100, 0.97, 600, 16, True), (150, 4, 2048, 1.0, 1900, 0, False),
+    (75, 8, 2500, 0.99, 0, 0, False), (75, 8, 1024, 0.995, 0, 0, True),
 ]
 
 
@@ -212,8 +213,11 @@ def test_kv_compress_bit_exact(case):
     if use_range:
         e_lo = r.integers(0, cap // 4, size=B).astype(np.int32)
         e_hi = (e_lo + cap // 2).astype(np.int32)
-    want = O.kv_compress(f64(Kc), f64(Vc), acc, ln, e_lo=e_lo, e_hi=e_hi, beta=beta,
-                         budget=budget if budget > 0 else None, recent=recent, pos=pos)
+    # with hundreds of heads (the shapes that get one warp per head) the oracle checks three of the sequences
+    sel = np.array([0, B // 2, B - 1]) if B * Hkv >= 500 else np.arange(B)
+    want = O.kv_compress(f64(Kc[sel]), f64(Vc[sel]), acc[sel], ln[sel], e_lo=None if e_lo is None else e_lo[sel],
+                         e_hi=None if e_hi is None else e_hi[sel], beta=beta,
+                         budget=budget if budget > 0 else None, recent=recent, pos=pos[sel])
     Kd, Vd = Kc.cuda(), Vc.cuda()
     ad, ld, pd = torch.from_numpy(acc).cuda(), torch.from_numpy(ln).cuda(), torch.from_numpy(pos).cuda()
     flag = status_tensor()
@@ -222,9 +226,10 @@ def test_kv_compress_bit_exact(case):
                   e_hi=None if e_hi is None else torch.from_numpy(e_hi).cuda())
     torch.cuda.synchronize()
     assert flag.item() == 0
-    assert np.array_equal(i32(ld), want["len"])
-    gK, gV, ga, gp = f64(Kd), f64(Vd), ad.cpu().numpy(), i32(pd)
-    for b in range(B):
+    assert np.array_equal(i32(ld)[sel], want["len"])
+    sel_d = torch.from_numpy(sel).cuda()
+    gK, gV, ga, gp = f64(Kd[sel_d]), f64(Vd[sel_d]), ad[sel_d].cpu().numpy(), i32(pd[sel_d])
+    for b in range(len(sel)):
         for g in range(Hkv):
             m = want["len"][b, g]
             assert np.array_equal(gK[b, g, :m], want["Kc"][b, g, :m].astype(np.float64)), (b, g)
