@@ -26,6 +26,7 @@ constexpr int kStreamThreads = kHidThreads + 64;   // ... plus the warps that is
 constexpr int kHidMaxChunks = 4;       // column groups per thread: rows up to 4 * 256 * 8 = 8192 channels
 constexpr int kNoRow = -2147483647 - 1;  // marks a slot of a tile that holds no row
 constexpr int kHidCluster = 8;         // CTAs whose partial sums are added through shared memory
+constexpr int kMaxHidPartials = 80;    // partial rows of a sequence the launch accepts when it makes the clusters smaller
 constexpr int kStreamMaxStages = 16;   // tiles in flight per CTA
 constexpr int kStreamRingBytes = 172 * 1024;  // shared-memory ring of a CTA (one CTA per SM)
 constexpr int kStreamTileBytes = 34 * 1024;   // rows are grouped into tiles of about this size
@@ -86,7 +87,10 @@ static bool merge_layout(const lvlm_dims* d, MergeLayout* L) {
     L->off_dst = off;     off = align_up(off + (size_t)d->B * d->N * 4, 256);
     L->off_wgt = off;     off = align_up(off + (size_t)d->B * d->n * 4, 256);
     L->off_meta = off;    off = align_up(off + (size_t)d->B * kMetaInts * 4, 256);
-    L->off_partial = off; off = align_up(off + (size_t)d->B * (cps / L->grid.cl) * d->C * 4, 256);
+    // (the launch may settle for smaller clusters than grid.cl, up to kMaxHidPartials partial rows a sequence)
+    const int few = cps < kMaxHidPartials ? cps : kMaxHidPartials;
+    const int prow = cps / L->grid.cl > few ? cps / L->grid.cl : few;
+    L->off_partial = off; off = align_up(off + (size_t)d->B * prow * d->C * 4, 256);
     L->off_kvpartial = off;
     if (d->Hkv > 0) off = align_up(off + (size_t)d->B * d->Hkv * 2 * L->kvP * kHeadDim * 4, 256);
     L->total = off;
@@ -665,27 +669,35 @@ lvlm_status launch_hidden_rows(const void* hidden, void* hidden_out, int64_t hid
                                int* partials_out) {
     const int chunks = (L.V + kHidThreads - 1) / kHidThreads;
     if (chunks > kHidMaxChunks || L.nstage < 3) return LVLM_ERR_UNSUPPORTED;  // more than 8192 channels
-    // no more clusters than the device runs at a time: a second wave would double the time
-    int resident = 0;
-    switch (chunks) {
-        case 1: resident = stream_clusters_resident<1>(L.cl); break;
-        case 2: resident = stream_clusters_resident<2>(L.cl); break;
-        case 3: resident = stream_clusters_resident<3>(L.cl); break;
-        case 4: resident = stream_clusters_resident<4>(L.cl); break;
+    // No more clusters than the device runs at a time: a second wave would double the time.  Clusters are placed
+    // inside one GPC, so large clusters leave SMs idle: the cluster size is halved while that puts more CTAs to work
+    // and the partial rows of a sequence stay few.
+    int cps = 0, cl_run = L.cl;
+    for (int cl = L.cl; cl >= 1; cl >>= 1) {
+        int resident = 0;
+        switch (chunks) {
+            case 1: resident = stream_clusters_resident<1>(cl); break;
+            case 2: resident = stream_clusters_resident<2>(cl); break;
+            case 3: resident = stream_clusters_resident<3>(cl); break;
+            case 4: resident = stream_clusters_resident<4>(cl); break;
+        }
+        int c = L.cps / cl * cl;
+        if (resident > 0) {
+            int per_seq = resident / d->B;
+            per_seq = per_seq < 1 ? 1 : per_seq;
+            if (c > per_seq * cl) c = per_seq * cl;
+        }
+        // (not for short sequences: there the extra partial rows cost more than the idle SMs)
+        if (cl < L.cl && (c / cl > kMaxHidPartials || d->N < 48 * L.cps)) break;
+        if (c > cps) { cps = c; cl_run = cl; }
     }
-    int cps = L.cps;
-    if (resident > 0) {
-        int per_seq = resident / d->B;
-        per_seq = per_seq < 1 ? 1 : per_seq;
-        if (cps > per_seq * L.cl) cps = per_seq * L.cl;
-    }
-    if (partials_out) *partials_out = cps / L.cl;
+    if (partials_out) *partials_out = cps / cl_run;
     StreamArgs a;
     a.hid = static_cast<const char*>(hidden);
     a.out = static_cast<char*>(hidden_out);
     a.scratch = static_cast<char*>(scratch);
     a.hid_sb = hid_sb * 2; a.out_sb = out_sb * 2; a.scr_sb = scr_sb * 2;
-    a.rowB = d->C * 2; a.V = L.V; a.N = d->N; a.i0 = d->i0; a.n = d->n; a.k = d->k; a.cl = L.cl;
+    a.rowB = d->C * 2; a.V = L.V; a.N = d->N; a.i0 = d->i0; a.n = d->n; a.k = d->k; a.cl = cl_run;
     a.rpt = L.rpt; a.slotB = L.slotB; a.nstage = L.nstage;
     a.dst_map = dst_map; a.wgt = wgt; a.meta = meta; a.partial = partial;
     a.K = nullptr; a.Vc = nullptr; a.kv_sb = a.kv_sh = 0; a.Hkv = 0; a.kvP = 1; a.kvL = 1; a.kvT = 16;
@@ -699,10 +711,10 @@ lvlm_status launch_hidden_rows(const void* hidden, void* hidden_out, int64_t hid
     }
     a.dev_status = dev_status;
     switch (chunks) {
-        case 1: return launch_row_stream<1>(a, cps, L.cl, d->B, stream);
-        case 2: return launch_row_stream<2>(a, cps, L.cl, d->B, stream);
-        case 3: return launch_row_stream<3>(a, cps, L.cl, d->B, stream);
-        case 4: return launch_row_stream<4>(a, cps, L.cl, d->B, stream);
+        case 1: return launch_row_stream<1>(a, cps, cl_run, d->B, stream);
+        case 2: return launch_row_stream<2>(a, cps, cl_run, d->B, stream);
+        case 3: return launch_row_stream<3>(a, cps, cl_run, d->B, stream);
+        case 4: return launch_row_stream<4>(a, cps, cl_run, d->B, stream);
     }
     return LVLM_ERR_UNSUPPORTED;
 }
