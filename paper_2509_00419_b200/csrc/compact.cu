@@ -28,7 +28,7 @@ constexpr int kIdxPerThread = 2;             // positions of a super-tile per th
 struct InplaceArgs {
     char* base0; char* base1;
     int64_t stride_b, stride_g, map_stride;
-    int G, T, V, Vsub, S, Nout, meta_stride, maps_per_g, Rmax, CG, RL, merged_row, P;
+    int G, T, V, Vsub, S, Nout, meta_stride, maps_per_g, Rmax, CG, RL, merged_row, P, early;
     const int32_t* src_map; const int32_t* meta; const int32_t* nout; const float* partial;
     char* fin_base; int64_t fin_stride_b; int fin_row, fin_V, fin_P, fin_y; const float* fin_partial;
     uint32_t* side_dst[2]; const uint32_t* side_src[2];
@@ -83,8 +83,9 @@ __device__ __forceinline__ uint4 sum_partials(const float* pp, int P, int64_t ro
 template <int MAXC>                                      // 16-byte column groups per thread
 __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const InplaceArgs a) {
     extern __shared__ __align__(16) uint4 tile[];
-    pdl_enter();
+    if (!a.early) pdl_enter();
     if ((int)blockIdx.y == a.fin_y) {                    // merged row of the other tensor: the CTAs of this row share its columns
+        if (a.early) pdl_enter();
         const int b = blockIdx.z;
         const float* pp = a.fin_partial + (int64_t)b * a.fin_P * a.fin_V * 8;
         uint4* out = reinterpret_cast<uint4*>(a.fin_base + (int64_t)b * a.fin_stride_b) + (int64_t)a.fin_row * a.fin_V;
@@ -164,6 +165,7 @@ __global__ void __launch_bounds__(kCompactThreads) inplace_compact_kernel(const 
         __syncthreads();
     }
     load_tile(0, buf[0]);
+    if (a.early) pdl_enter();                         // the partial rows and every write come after the kernel ahead
     int k = 0;
     for (int t0 = o_start; t0 < Nout; t0 += Rc, ++k) {
         if (t0 + Rc < Nout) load_tile((k + 1) % 3, buf[(k + 1) & 1]);
@@ -220,6 +222,7 @@ lvlm_status launch_inplace_compact(const CompactJob& j, cudaStream_t stream) {
     a.map_stride = j.map_stride > 0 ? j.map_stride : j.N;
     a.src_map = j.src_map; a.meta = j.meta; a.nout = j.nout;
     a.merged_row = j.merged_row; a.partial = j.partial; a.P = j.P;
+    a.early = j.maps_ready && !j.side_dst[0] && !j.side_dst[1] ? 1 : 0;
     if (fin) a.fin_y = j.G * a.T;
     for (int i = 0; i < 2; ++i) {
         a.side_dst[i] = static_cast<uint32_t*>(j.side_dst[i]);

@@ -34,6 +34,10 @@ struct CompactJob {
     // Optionally, in the same launch: row `fin_row` of every sequence of another tensor (rows of fin_V 16-byte
     // vectors, sequences fin_stride_b bytes apart) receives the sum of the fin_P partial rows
     // fin_partial[(b*fin_P + p)*fin_V*8 ...].  base0 may be NULL then: nothing is compacted.
+    // The maps, meta and nout were complete, and the rows were no longer written, before the kernel ahead of this
+    // launch in the stream let it start (that kernel only reads the rows): the first rows are then fetched while it
+    // still runs; the partial rows and every write wait for it.
+    bool maps_ready = false;
     void* fin_base = nullptr;
     int64_t fin_stride_b = 0;
     int fin_row = 0, fin_V = 0, fin_P = 0;

@@ -360,9 +360,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) row_stream_kernel(const Str
     __syncthreads();
     // The kernel ahead in the stream (the plan) writes the row maps and weights only, and it has itself waited for
     // everything before it: the rows can be fetched while it still runs.  The loader does so for the first lap of
-    // the ring before it waits; every other warp waits here.
-    if (warp != kLoaderWarp) pdl_wait();
-    pdl_launch_dependents();
+    // the ring before it waits; every other warp waits here.  Nobody lets the next kernel start before it has
+    // waited itself: that kernel may then take the plan for complete as soon as it runs.
+    if (warp != kLoaderWarp) { pdl_wait(); pdl_launch_dependents(); }
 
     const int32_t* dst = a.dst_map + (int64_t)b * a.N;
     const float* w = a.wgt ? a.wgt + (int64_t)b * a.n - a.i0 : nullptr;     // indexed by sequence position
@@ -455,6 +455,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) row_stream_kernel(const Str
         // whole-tile copies need no table: the first lap of the ring starts before the wait
         for (; more && j < S && (t.kv || a.out); ++j, ++slot) { fetch(t, slot, j); more = it.next(&t); }
         pdl_wait();
+        pdl_launch_dependents();
         for (int q = 0; q < j + kTabAhead; ++q) request_table();
         asm volatile("cp.async.wait_group %0;\n" ::"n"(kTabAhead) : "memory");          // the tables of the tiles under way
         __syncwarp();
@@ -811,7 +812,7 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
         j.base0 = hidden; j.stride_b = hid_sb * 2; j.B = d->B; j.G = 1; j.V = L.V;
         j.src_map = src_map; j.map_stride = d->N; j.meta = meta; j.meta_stride = kMetaInts;
         j.Nout = L.Nout; j.N = d->N; j.merged_row = d->i0 + d->k; j.partial = partial;
-        j.P = hid_partials;
+        j.P = hid_partials; j.maps_ready = true;
         const lvlm_status st = launch_inplace_compact(j, stream);
         if (st != LVLM_OK) return st;
     }
@@ -826,7 +827,7 @@ extern "C" lvlm_status lvlm_merge_compact(void* hidden, void* hidden_out, void* 
         j.src_map = src_map; j.map_stride = d->N; j.meta = meta; j.meta_stride = kMetaInts;
         j.Nout = L.Nout; j.merged_row = d->i0 + d->k; j.partial = kv_partial; j.P = L.kvP;
     }
-    j.B = d->B; j.N = d->N;
+    j.B = d->B; j.N = d->N; j.maps_ready = true;
     if (Kc || hidden_out) {
         const lvlm_status st = launch_inplace_compact(j, stream);
         if (st != LVLM_OK) return st;
