@@ -131,7 +131,8 @@ __device__ __forceinline__ uint32_t stage_off(int r, int ch) {
 }
 
 // grid.x = heads * S, clusters of S CTAs along x: cluster = (sequence, KV head), rank = run of tiles.
-template <int G>
+// CL = false: one CTA per head and no cluster instruction in the kernel at all.
+template <int G, bool CL>
 __global__ void __launch_bounds__(kDecThreads, 2)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                       const DecodeArgs a) {
@@ -162,9 +163,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     // With a.early the first key/value stages and the length are fetched while the kernel ahead in the
     // stream is still finishing; q, k_new, v_new and every write come after the wait in any case.
     if (!a.early) pdl_enter();
-    const int S = a.S, H = a.H, cap = a.cap;
+    const int S = CL ? a.S : 1, H = a.H, cap = a.cap;
     const int hd = blockIdx.x / S;
-    const int rank = (int)cluster_ctarank();
+    const int rank = CL ? (int)cluster_ctarank() : 0;
     const int b = hd / a.Hkv, g = hd % a.Hkv, h0 = g * G;
 
     // ---- this head's length; every CTA of the cluster takes the same decisions ---------------------------
@@ -404,7 +405,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     }
 
     // ---- combine the CTAs of the cluster in rank order through distributed shared memory ----------------
-    cluster_sync_all();
+    if (CL) cluster_sync_all(); else __syncthreads();
     // my slice of the output channels: element (hh, d) with hh*128 + d = rank*128 + tid (+ S*128 ...).
     // A thread fetches what it needs from every CTA in one go (max, sum and its channel) and
     // works out the weights itself, so there is one round trip and no block barrier on this path.
@@ -418,9 +419,13 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         for (int r = 0; r < kDecMaxCluster; ++r) {
             x[r] = 0.f; m[r] = -INFINITY; l[r] = 0.f;
             if (r < S) {
-                x[r] = dsmem_ld(dsmem_addr(a_o, r));
-                m[r] = dsmem_ld(dsmem_addr(a_m, r));
-                l[r] = dsmem_ld(dsmem_addr(a_l, r));
+                if (CL) {
+                    x[r] = dsmem_ld(dsmem_addr(a_o, r));
+                    m[r] = dsmem_ld(dsmem_addr(a_m, r));
+                    l[r] = dsmem_ld(dsmem_addr(a_l, r));
+                } else {                       // a head with one CTA: its own shared memory, read directly
+                    x[r] = s_acc[idx]; m[r] = s_M[hh]; l[r] = s_L[hh];
+                }
             }
         }
         float FM = -INFINITY;
@@ -435,7 +440,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         }
         a.out[(int64_t)(b * H + h0) * kHeadDim + idx] = __float2bfloat16_rn(Ls > 0.f ? v / Ls : 0.f);
     }
-    if (a.acc_score && tid < 8 * S) {          // (max, sum) of every CTA and head, for the acc_score update
+    if (CL && a.acc_score && tid < 8 * S) {    // (max, sum) of every CTA and head, for the acc_score update
         const int r = tid >> 3, hh = tid & 7;
         float m = -INFINITY, l = 0.f;
         if (hh < G) {
@@ -445,11 +450,15 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         s_rm[tid] = m;
         s_rl[tid] = l;
     }
-    cluster_arrive();                          // my reads of the other CTAs' shared memory are done
+    if (CL) cluster_arrive();                  // my reads of the other CTAs' shared memory are done
     // the probabilities of my own keys go to acc_score
     if (a.acc_score) {
-        __syncthreads();
-        if (tid < G) {
+        if (!CL) {                             // one CTA: its own (max, sum) are the head's
+            if (tid < G) { s_FM[tid] = s_M[tid]; s_FI[tid] = s_L[tid] > 0.f ? 1.0f / s_L[tid] : 0.f; }
+        } else {
+            __syncthreads();
+        }
+        if (CL && tid < G) {
             float FM = -INFINITY;
             for (int r = 0; r < S; ++r) FM = fmaxf(FM, s_rm[r * 8 + tid]);
             float Ls = 0.f;
@@ -494,7 +503,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         }
     }
     if (app && rank == 0 && tid == 0) a.len[hd] = lne;    // every CTA of the cluster read it before the barrier
-    cluster_wait();                                       // nobody leaves while its shared memory is still read
+    if (CL) cluster_wait();                               // nobody leaves while its shared memory is still read
 }
 
 template <int G>
@@ -510,7 +519,9 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
     const int logit_keys = acc_score && (size_t)G * run_keys * 4 <= (size_t)kDecLogitBytes ? run_keys : 0;
     const size_t smem = 1024 + (size_t)kRingBytes + (size_t)(2 * kDecWarps * 8 + 4 * 8 + 2 * 8 * kDecMaxCluster) * 4 +
                         (size_t)(2 * kStagesDec + 1) * 8 + (size_t)G * logit_keys * 4;
-    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(decode_cluster_kernel<G>,
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(decode_cluster_kernel<G, true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+    LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(decode_cluster_kernel<G, false>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
     CUtensorMap kmap, vmap;
     {
@@ -538,7 +549,9 @@ static lvlm_status launch_decode(const void* q, void* Kc, void* Vc, int32_t* len
     a.logit_keys = logit_keys;
     a.dev_status = dev_status;
 
-    return launch_kernel(decode_cluster_kernel<G>, dim3((unsigned)ctas), dim3(kDecThreads), smem, stream, L.S, kmap, vmap, a);
+    if (L.S == 1)
+        return launch_kernel(decode_cluster_kernel<G, false>, dim3((unsigned)ctas), dim3(kDecThreads), smem, stream, 1, kmap, vmap, a);
+    return launch_kernel(decode_cluster_kernel<G, true>, dim3((unsigned)ctas), dim3(kDecThreads), smem, stream, L.S, kmap, vmap, a);
 }
 
 }  // namespace lvlm
