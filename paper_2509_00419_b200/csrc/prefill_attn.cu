@@ -4,16 +4,20 @@
 //
 // One CTA per (sequence, query head, tile of 128 query rows); tcgen05 MMAs, accumulators in tensor memory:
 //   S = Q K_j^T      A = Q tile, B = K tile, both K-major from TMA (128-byte swizzle), 128x128 fp32 in TMEM (two
-//                    buffers: the next tile is multiplied while this one is in the softmax)
-//   softmax          four warps, thread = query row (TMEM lane): running max m and sum l in the log2 domain; the
-//                    probabilities 2^(s - m) go to shared memory as bf16 (head and remainder, two planes) in the
-//                    K-major swizzled layout; the output
-//                    accumulator is rescaled only when the maximum has grown by more than 2^8 (the stale maximum
-//                    keeps every probability below 2^8, well inside bf16 and fp32)
-//   O += P V_j       A = P from shared memory, B = V tile as it lies in memory (keys x channels: an MN-major
-//                    operand), 128x128 fp32 in TMEM
-// At the end a thread divides its row by l, writes it, writes lse = ln sum exp of the row, and - for the rows of
-// the scoring window - the log2-domain normaliser the column-sum pass of lvlm_score_tokens reads; that pass then
+//                    buffers: the tile after next is multiplied while this one is in the softmax)
+//   softmax          eight warps: thread = (query row, half of the tile's 128 keys); the row maximum of a tile meets
+//                    in shared memory (one named barrier a tile); running max m and sum l in the log2 domain.  The
+//                    probabilities 2^(s - m) go back into the tensor-memory columns the logits came from, as
+//                    bf16 pairs (head and remainder of every probability: a plain bf16 would miss the output
+//                    tolerance on rows that see few keys), so P never touches shared memory and the buffer of a
+//                    tile holds first its S, then its P.  The output accumulator is rescaled only when the maximum
+//                    has grown by more than 2^8 (the stale maximum keeps every probability below 2^8, well inside
+//                    bf16 and fp32), and only then does the softmax wait for the product before it
+//   O += P V_j       A = P from tensor memory, B = V tile as it lies in memory (keys x channels: an MN-major
+//                    operand), 128x128 fp32 in TMEM; the MMAs of one thread run in the order of issue, so the
+//                    next S may be written over a P that an earlier MMA still reads
+// At the end a thread divides its half row by l, writes it, writes lse = ln sum exp of the row, and - for the rows
+// of the scoring window - the log2-domain normaliser the column-sum pass of lvlm_score_tokens reads; that pass then
 // runs on the same stream (keys on the TMEM lanes, see score_tc.cu) and produces score and score_head.
 #include "common.cuh"
 #include "score.cuh"
@@ -26,9 +30,10 @@ using namespace sm100;
 constexpr int kAT = 128;                     // query rows per CTA, keys per tile, head dim
 constexpr int kAHalf = kAT * 64 * 2;         // one TMA box: 128 rows x 64 bf16 = 16 KB
 constexpr int kATile = 2 * kAHalf;           // 32 KB
-constexpr int kAStages = 2;                  // K/V ring
-constexpr int kAThreads = 192;               // warp 0 TMA, warp 1 MMA, warps 2..5 softmax
-constexpr uint32_t kATmemCols = 512;         // S0 | S1 | O | (unused)
+constexpr int kAStages = 2;                  // K ring and V ring (released separately: K after S, V after O)
+constexpr int kASoftmaxThreads = 256;        // warps 2..9
+constexpr int kAThreads = 64 + kASoftmaxThreads;   // warp 0 TMA, warp 1 MMA
+constexpr uint32_t kATmemCols = 512;         // S0/P0 | S1/P1 | O | (unused)
 constexpr float kLog2eA = 1.4426950408889634f;
 constexpr float kLn2A = 0.6931471805599453f;
 constexpr float kRescaleStep = 8.0f;         // the output is rescaled when the row maximum has grown by more (log2)
@@ -43,10 +48,22 @@ struct AttnArgs {
 };
 
 struct AttnSmem {
-    uint64_t q_full, kv_full[kAStages], kv_empty[kAStages], s_full[2], s_empty[2], p_ready, o_done;
+    uint64_t q_full, k_full[kAStages], k_empty[kAStages], v_full[kAStages], v_empty[kAStages], s_full[2], p_ready, o_done;
     uint32_t tmem_base;
     volatile int abort;
+    float xmax[2][2][kAT];     // [tile parity][half][row]: the tile maximum of a half row, for the other half
+    float xl[kAT];             // the sum of the upper half row, for the thread that writes lse
 };
+
+// D[tmem] (+)= A[tmem] * B[smem]^T, issued by one thread: A is 128 rows (lanes) of bf16 pairs, two K indices a column.
+__device__ __forceinline__ void mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 
 // Shared-memory descriptor of an MN-major bf16 operand stored as rows of 128 bytes (64 elements of the M or N
 // dimension) with the 128-byte swizzle, one row per K index: 8 rows are one swizzle atom (stride byte offset 1024
@@ -100,9 +117,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
     unsigned char* sQ = base;
     unsigned char* sK = base + kATile;                            // [kAStages] tiles
     unsigned char* sV = sK + kAStages * kATile;                   // [kAStages] tiles
-    unsigned char* sP = sV + kAStages * kATile;                   // bf16 probabilities ...
-    unsigned char* sP2 = sP + kATile;                             // ... and what bf16 rounding left of them
-    AttnSmem* sm = reinterpret_cast<AttnSmem*>(sP2 + kATile);
+    AttnSmem* sm = reinterpret_cast<AttnSmem*>(sV + kAStages * kATile);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x, h = blockIdx.y, b = blockIdx.z, g = h / a.G;
@@ -112,9 +127,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
 
     if (threadIdx.x == 0) {
         mbar_init(&sm->q_full, 1);
-        for (int s = 0; s < kAStages; ++s) { mbar_init(&sm->kv_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sm->s_full[s], 1); mbar_init(&sm->s_empty[s], kAT); }
-        mbar_init(&sm->p_ready, kAT);
+        for (int s = 0; s < kAStages; ++s) {
+            mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
+            mbar_init(&sm->v_full[s], 1); mbar_init(&sm->v_empty[s], 1);
+        }
+        for (int s = 0; s < 2; ++s) mbar_init(&sm->s_full[s], 1);
+        mbar_init(&sm->p_ready, kASoftmaxThreads);
         mbar_init(&sm->o_done, 1);
         sm->abort = 0;
         fence_barrier_init();
@@ -139,12 +157,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
             tma_load_4d(sQ + kAHalf, &qmap, &sm->q_full, 64, h, qt * kAT, b);
             for (int j = 0; j < nk; ++j) {
                 const int st = j % kAStages;
-                if (j >= kAStages && !attn_wait(&sm->kv_empty[st], ((j / kAStages) - 1) & 1, sm, a.dev_status)) break;
-                mbar_arrive_expect_tx(&sm->kv_full[st], 2 * kATile);
-                tma_load_4d(sK + st * kATile, &kmap, &sm->kv_full[st], 0, j * kAT, g, b);
-                tma_load_4d(sK + st * kATile + kAHalf, &kmap, &sm->kv_full[st], 64, j * kAT, g, b);
-                tma_load_4d(sV + st * kATile, &vmap, &sm->kv_full[st], 0, j * kAT, g, b);
-                tma_load_4d(sV + st * kATile + kAHalf, &vmap, &sm->kv_full[st], 64, j * kAT, g, b);
+                if (j >= kAStages && !attn_wait(&sm->k_empty[st], ((j / kAStages) - 1) & 1, sm, a.dev_status)) break;
+                mbar_arrive_expect_tx(&sm->k_full[st], kATile);
+                tma_load_4d(sK + st * kATile, &kmap, &sm->k_full[st], 0, j * kAT, g, b);
+                tma_load_4d(sK + st * kATile + kAHalf, &kmap, &sm->k_full[st], 64, j * kAT, g, b);
+                if (j >= kAStages && !attn_wait(&sm->v_empty[st], ((j / kAStages) - 1) & 1, sm, a.dev_status)) break;
+                mbar_arrive_expect_tx(&sm->v_full[st], kATile);
+                tma_load_4d(sV + st * kATile, &vmap, &sm->v_full[st], 0, j * kAT, g, b);
+                tma_load_4d(sV + st * kATile + kAHalf, &vmap, &sm->v_full[st], 64, j * kAT, g, b);
             }
         }
     } else if (warp == 1) {
@@ -152,68 +172,77 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc_qk = idesc_bf16_f32(kAT, kAT);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kAT, kAT) | (1u << 16);     // B (the V tile) is MN-major
-            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP), p2_addr = smem_u32(sP2);
-            auto issue_qk = [&](int j) {
-                const uint32_t k_addr = smem_u32(sK + (j % kAStages) * kATile);
+            const uint32_t q_addr = smem_u32(sQ);
+            // S_j into buffer j & 1 (over P_{j-2}: the MMAs that read it were issued before this one)
+            auto issue_qk = [&](int j) -> bool {
+                const int st = j % kAStages;
+                if (!attn_wait(&sm->k_full[st], (j / kAStages) & 1, sm, a.dev_status)) return false;
+                tc_fence_after();
+                const uint32_t k_addr = smem_u32(sK + st * kATile);
                 const uint32_t d_tmem = tmem_base + (j & 1) * kAT;
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const uint32_t off = (k >> 2) * kAHalf + (k & 3) * 32;
                     mma_bf16_ss(d_tmem, smem_desc_sw128(q_addr + off), smem_desc_sw128(k_addr + off), idesc_qk, k > 0);
                 }
+                mma_commit(&sm->k_empty[st]);              // the K tile may be refilled once these are done
                 mma_commit(&sm->s_full[j & 1]);
+                return true;
             };
             bool ok = attn_wait(&sm->q_full, 0, sm, a.dev_status);
-            if (ok) ok = attn_wait(&sm->kv_full[0], 0, sm, a.dev_status);
-            if (ok) { tc_fence_after(); issue_qk(0); }
+            if (ok && nk > 0) ok = issue_qk(0);
+            if (ok && nk > 1) ok = issue_qk(1);
             for (int j = 0; ok && j < nk; ++j) {
-                if (j + 1 < nk) {                            // the next tile's logits while this one is in the softmax
-                    ok = attn_wait(&sm->kv_full[(j + 1) % kAStages], ((j + 1) / kAStages) & 1, sm, a.dev_status);
-                    if (ok && j + 1 >= 2) ok = attn_wait(&sm->s_empty[(j + 1) & 1], (((j + 1) / 2) - 1) & 1, sm, a.dev_status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(j + 1);
-                }
                 ok = attn_wait(&sm->p_ready, j & 1, sm, a.dev_status);
+                if (ok) ok = attn_wait(&sm->v_full[j % kAStages], (j / kAStages) & 1, sm, a.dev_status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t v_addr = smem_u32(sV + (j % kAStages) * kATile);
+                const uint32_t p_tmem = tmem_base + (j & 1) * kAT;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {               // 16 keys per step
-                    const uint32_t aoff = (k >> 2) * kAHalf + (k & 3) * 32;
+                for (int k = 0; k < 8; ++k) {               // 16 keys per step: 8 columns of bf16 pairs
+                    const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;       // heads; the remainders lie 16 columns on
                     const uint64_t vdesc = smem_desc_mn_sw128(v_addr + k * 2048, kAHalf);
-                    mma_bf16_ss(tmem_o, smem_desc_sw128(p_addr + aoff), vdesc, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
-                    mma_bf16_ss(tmem_o, smem_desc_sw128(p2_addr + aoff), vdesc, idesc_pv, 1u);
+                    mma_bf16_ts(tmem_o, pa, vdesc, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+                    mma_bf16_ts(tmem_o, pa + 16, vdesc, idesc_pv, 1u);
                 }
-                mma_commit(&sm->kv_empty[j % kAStages]);    // K and V of this tile are done with
+                mma_commit(&sm->v_empty[j % kAStages]);     // the V tile is done with
                 mma_commit(&sm->o_done);
+                if (j + 2 < nk) ok = issue_qk(j + 2);       // the logits of the tile after next, while the next one is in the softmax
             }
         }
     } else {
-        // ================= softmax: thread = query row =================
-        const int quarter = warp & 3;
+        // ================= softmax: thread = (query row, half of the keys of a tile) =================
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
         const int pos = qt * kAT + row;                      // sequence position of my query
         const uint32_t lane_addr = ((uint32_t)(quarter * 32) << 16);
-        float m_used = -INFINITY, l_run = 0.f;
+        float m_used = -INFINITY, l_run = 0.f;               // l_run: the sum over my half of the keys
+        // Every thread runs every round and meets the others at the named barrier, also after a wait has given up
+        // (`ok`, the same for all lanes of a warp, then only switches the work off).
         bool ok = true;
         for (int j = 0; j < nk; ++j) {
             const int buf = j & 1;
-            ok = ok && attn_wait(&sm->s_full[buf], (j / 2) & 1, sm, a.dev_status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t s_addr = tmem_base + lane_addr + buf * kAT;
-            const int lim = min(a.N, a.causal ? pos + 1 : a.N) - j * kAT;     // keys j*128 + c with c < lim are visible
-            // first sweep: the row maximum of this tile
+            ok = __all_sync(0xFFFFFFFFu, ok && attn_wait(&sm->s_full[buf], (j / 2) & 1, sm, a.dev_status));
+            const uint32_t s_addr = tmem_base + lane_addr + buf * kAT + half * 64;
+            const int lim = min(a.N, a.causal ? pos + 1 : a.N) - j * kAT - half * 64;   // my columns c < lim are visible
+            float v[2][32];
             float tmax = -INFINITY;
-#pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-                float v[32];
-                tmem_ld32(s_addr + c4 * 32, v);
+            if (ok) {
+                tc_fence_after();
+                tmem_ld32(s_addr, v[0]);
+                tmem_ld32(s_addr + 32, v[1]);
                 tmem_ld_wait();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) tmax = fmaxf(tmax, c4 * 32 + c < lim ? v[c] : -INFINITY);
+                for (int c2 = 0; c2 < 2; ++c2)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) tmax = fmaxf(tmax, c2 * 32 + c < lim ? v[c2][c] : -INFINITY);
             }
+            // the maximum of the row's other half
+            sm->xmax[buf][half][row] = tmax;
+            asm volatile("bar.sync 1, %0;" ::"n"(kASoftmaxThreads) : "memory");
+            if (!ok) continue;
+            tmax = fmaxf(tmax, sm->xmax[buf][half ^ 1][row]);
             tmax *= a.scale_log2;                            // a positive scale keeps the order
             float corr = 1.f;
             bool grow = false;
@@ -222,83 +251,73 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
                 m_used = tmax;
                 grow = true;
             }
-            // the previous product has to be finished before P is overwritten or O is touched
-            if (j > 0) {
-                ok = attn_wait(&sm->o_done, (j - 1) & 1, sm, a.dev_status);
-                if (!ok) break;
+            // O is touched only when some row of the warp moves its reference: the products issued so far have to be done
+            if (j > 0 && __any_sync(0xFFFFFFFFu, grow)) {
+                ok = __all_sync(0xFFFFFFFFu, attn_wait(&sm->o_done, (j - 1) & 1, sm, a.dev_status));
+                if (!ok) continue;
                 tc_fence_after();
-                if (__any_sync(0xFFFFFFFFu, grow)) {
-                    l_run *= corr;
+                l_run *= corr;
 #pragma unroll 1
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        float o[32];
-                        tmem_ld32(tmem_o + lane_addr + c4 * 32, o);
-                        tmem_ld_wait();
+                for (int c2 = 0; c2 < 2; ++c2) {             // my half of the channels
+                    float o[32];
+                    tmem_ld32(tmem_o + lane_addr + half * 64 + c2 * 32, o);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] *= corr;
-                        tmem_st32(tmem_o + lane_addr + c4 * 32, o);
-                    }
-                    tmem_st_wait();
+                    for (int c = 0; c < 32; ++c) o[c] *= corr;
+                    tmem_st32(tmem_o + lane_addr + half * 64 + c2 * 32, o);
                 }
+                tmem_st_wait();
             }
-            // second sweep: probabilities relative to m_used, to shared memory as the A operand of P V
+            // probabilities relative to m_used, written over the logits they came from: 32 logits become 16 columns
+            // of bf16 pairs (the bf16 rounding of every probability) and 16 columns of what the rounding left
             const float mref = m_used == -INFINITY ? 0.f : m_used;
             float psum = 0.f;
-#pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-                float v[32];
-                tmem_ld32(s_addr + c4 * 32, v);
-                tmem_ld_wait();
-                // a probability is split into its bf16 rounding and a bf16 of the rest, so that the product with V
-                // keeps about 16 bits (rows that see few keys would otherwise miss the output tolerance)
-                uint32_t pk[16], pr[16];
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2) {
+                uint32_t pk[32];
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
-                    const float p0 = c4 * 32 + c < lim ? ex2_approx(fmaf(v[c], a.scale_log2, -mref)) : 0.f;
-                    const float p1 = c4 * 32 + c + 1 < lim ? ex2_approx(fmaf(v[c + 1], a.scale_log2, -mref)) : 0.f;
+                    const float p0 = c2 * 32 + c < lim ? ex2_approx(fmaf(v[c2][c], a.scale_log2, -mref)) : 0.f;
+                    const float p1 = c2 * 32 + c + 1 < lim ? ex2_approx(fmaf(v[c2][c + 1], a.scale_log2, -mref)) : 0.f;
                     pk[c >> 1] = pack_bf16(p0, p1);
-                    pr[c >> 1] = pack_bf16(p0 - bf16_lo(pk[c >> 1]), p1 - bf16_hi(pk[c >> 1]));
+                    pk[16 + (c >> 1)] = pack_bf16(p0 - bf16_lo(pk[c >> 1]), p1 - bf16_hi(pk[c >> 1]));
                     psum += p0 + p1;
                 }
-                // keys c4*32 .. +31 of my row: four 16-byte chunks of the 64-key half c4/2
-                const int poff = (c4 >> 1) * kAHalf + row * 128;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int chunk = (c4 & 1) * 4 + q;
-                    *reinterpret_cast<uint4*>(sP + poff + ((chunk ^ (row & 7)) << 4)) =
-                        make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-                    *reinterpret_cast<uint4*>(sP2 + poff + ((chunk ^ (row & 7)) << 4)) =
-                        make_uint4(pr[4 * q], pr[4 * q + 1], pr[4 * q + 2], pr[4 * q + 3]);
-                }
+                tmem_st32(s_addr + c2 * 32, reinterpret_cast<const float*>(pk));
             }
             l_run += psum;
+            tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(&sm->s_empty[buf]);                 // the logits of this buffer have been read
-            fence_proxy_async();                            // P is visible to the tensor core's reads
             mbar_arrive(&sm->p_ready);
         }
         // ---- the output row --------------------------------------------------------------------------------
-        if (ok && nk > 0) ok = attn_wait(&sm->o_done, (nk - 1) & 1, sm, a.dev_status);
+        ok = __all_sync(0xFFFFFFFFu, ok && (nk == 0 || attn_wait(&sm->o_done, (nk - 1) & 1, sm, a.dev_status)));
         tc_fence_after();
+        if (half == 1) sm->xl[row] = l_run;
+        asm volatile("bar.sync 1, %0;" ::"n"(kASoftmaxThreads) : "memory");
         {
+            const float l_row = half == 0 ? l_run + sm->xl[row] : 0.f;
+            if (half == 0) sm->xl[row] = l_row;
+            asm volatile("bar.sync 1, %0;" ::"n"(kASoftmaxThreads) : "memory");
+            const float l_all = sm->xl[row];
             const bool valid = ok && pos < a.N && !sm->abort;
-            const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-            __nv_bfloat16* orow = a.out + (int64_t)b * a.out_sb + (int64_t)pos * a.out_sn + (int64_t)h * a.out_sh;
+            const float inv = l_all > 0.f ? 1.0f / l_all : 0.f;
+            __nv_bfloat16* orow = a.out + (int64_t)b * a.out_sb + (int64_t)pos * a.out_sn + (int64_t)h * a.out_sh + half * 64;
 #pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {                // (the loads are warp-wide: every lane takes part)
+            for (int c2 = 0; c2 < 2; ++c2) {                // (the loads are warp-wide: every lane takes part)
                 float o[32];
-                tmem_ld32(tmem_o + lane_addr + c4 * 32, o);
+                tmem_ld32(tmem_o + lane_addr + half * 64 + c2 * 32, o);
                 tmem_ld_wait();
                 if (valid) {
-                    uint4* dst = reinterpret_cast<uint4*>(orow + c4 * 32);
+                    uint4* dst = reinterpret_cast<uint4*>(orow + c2 * 32);
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
                         dst[q] = make_uint4(pack_bf16(o[8 * q] * inv, o[8 * q + 1] * inv), pack_bf16(o[8 * q + 2] * inv, o[8 * q + 3] * inv),
                                             pack_bf16(o[8 * q + 4] * inv, o[8 * q + 5] * inv), pack_bf16(o[8 * q + 6] * inv, o[8 * q + 7] * inv));
                 }
             }
-            if (valid) {
-                const float lse2 = m_used + log2f(l_run);   // log2 of the row's sum of 2^(scaled logits)
+            if (valid && half == 0) {
+                const float lse2 = m_used + log2f(l_all);   // log2 of the row's sum of 2^(scaled logits)
                 a.lse[((int64_t)b * a.H + h) * a.N + pos] = lse2 * kLn2A;
                 if (a.lse_win && pos >= a.q_lo && pos < a.q_hi)
                     a.lse_win[((int64_t)b * a.H + h) * (a.q_hi - a.q_lo) + (pos - a.q_lo)] = lse2;
@@ -372,7 +391,7 @@ extern "C" lvlm_status lvlm_prefill_attn(const void* Q, const void* K, const voi
     a.lse = lse;
     a.lse_win = score ? reinterpret_cast<float*>(wsb + L.off_lse) : nullptr;
     a.dev_status = dev_status;
-    const size_t smem = 1024 + (size_t)kATile * (3 + 2 * kAStages) + sizeof(AttnSmem);
+    const size_t smem = 1024 + (size_t)kATile * (1 + 2 * kAStages) + sizeof(AttnSmem);
     LVLM_RETURN_IF_CUDA(cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int nqt = (d->N + kAT - 1) / kAT;
     lvlm_status s0 = launch_kernel(prefill_attn_kernel, dim3(nqt, d->H, d->B), dim3(kAThreads), smem, stream, 1,
