@@ -228,15 +228,27 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
             const int lim = min(a.N, a.causal ? pos + 1 : a.N) - j * kAT - half * 64;   // my columns c < lim are visible
             float v[2][32];
             float tmax = -INFINITY;
+            // off the diagonal every lane of the warp sees all of its 64 keys: no masks then
+            const bool full = __all_sync(0xFFFFFFFFu, lim >= 64);
             if (ok) {
                 tc_fence_after();
                 tmem_ld32(s_addr, v[0]);
                 tmem_ld32(s_addr + 32, v[1]);
                 tmem_ld_wait();
+                if (full) {
+                    float t0 = v[0][0], t1 = v[0][1], t2 = v[1][0], t3 = v[1][1];
 #pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2)
+                    for (int c = 2; c < 32; c += 2) {
+                        t0 = fmaxf(t0, v[0][c]); t1 = fmaxf(t1, v[0][c + 1]);
+                        t2 = fmaxf(t2, v[1][c]); t3 = fmaxf(t3, v[1][c + 1]);
+                    }
+                    tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
+                } else {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) tmax = fmaxf(tmax, c2 * 32 + c < lim ? v[c2][c] : -INFINITY);
+                    for (int c2 = 0; c2 < 2; ++c2)
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) tmax = fmaxf(tmax, c2 * 32 + c < lim ? v[c2][c] : -INFINITY);
+                }
             }
             // the maximum of the row's other half
             sm->xmax[buf][half][row] = tmax;
@@ -277,8 +289,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
                 uint32_t pk[32];
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
-                    const float p0 = c2 * 32 + c < lim ? ex2_approx(fmaf(v[c2][c], a.scale_log2, -mref)) : 0.f;
-                    const float p1 = c2 * 32 + c + 1 < lim ? ex2_approx(fmaf(v[c2][c + 1], a.scale_log2, -mref)) : 0.f;
+                    float p0 = ex2_approx(fmaf(v[c2][c], a.scale_log2, -mref));
+                    float p1 = ex2_approx(fmaf(v[c2][c + 1], a.scale_log2, -mref));
+                    if (!full) {
+                        p0 = c2 * 32 + c < lim ? p0 : 0.f;
+                        p1 = c2 * 32 + c + 1 < lim ? p1 : 0.f;
+                    }
                     pk[c >> 1] = pack_bf16(p0, p1);
                     pk[16 + (c >> 1)] = pack_bf16(p0 - bf16_lo(pk[c >> 1]), p1 - bf16_hi(pk[c >> 1]));
                     psum += p0 + p1;
