@@ -14,8 +14,8 @@
 //                    has grown by more than 2^8 (the stale maximum keeps every probability below 2^8, well inside
 //                    bf16 and fp32), and only then does the softmax wait for the product before it
 //   O += P V_j       A = P from tensor memory, B = V tile as it lies in memory (keys x channels: an MN-major
-//                    operand), 128x128 fp32 in TMEM; the MMAs of one thread run in the order of issue, so the
-//                    next S may be written over a P that an earlier MMA still reads
+//                    operand), 128x128 fp32 in TMEM; the next S is written into a buffer only when the product
+//                    that read its P is complete
 // At the end a thread divides its half row by l, writes it, writes lse = ln sum exp of the row, and - for the rows
 // of the scoring window - the log2-domain normaliser the column-sum pass of lvlm_score_tokens reads; that pass then
 // runs on the same stream (keys on the TMEM lanes, see score_tc.cu) and produces score and score_head.
@@ -173,7 +173,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
             constexpr uint32_t idesc_qk = idesc_bf16_f32(kAT, kAT);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kAT, kAT) | (1u << 16);     // B (the V tile) is MN-major
             const uint32_t q_addr = smem_u32(sQ);
-            // S_j into buffer j & 1 (over P_{j-2}: the MMAs that read it were issued before this one)
+            // S_j into buffer j & 1, over P_{j-2} (the caller has waited for the product that read it)
             auto issue_qk = [&](int j) -> bool {
                 const int st = j % kAStages;
                 if (!attn_wait(&sm->k_full[st], (j / kAStages) & 1, sm, a.dev_status)) return false;
@@ -208,7 +208,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
                 }
                 mma_commit(&sm->v_empty[j % kAStages]);     // the V tile is done with
                 mma_commit(&sm->o_done);
-                if (j + 2 < nk) ok = issue_qk(j + 2);       // the logits of the tile after next, while the next one is in the softmax
+                if (j + 2 < nk) {
+                    // The logits of the tile after next go where this tile's P lies: not before the product has read it
+                    // (the softmax of the next tile is far from done by then, so nothing waits for this wait).
+                    ok = attn_wait(&sm->o_done, j & 1, sm, a.dev_status);
+                    if (ok) ok = issue_qk(j + 2);
+                }
             }
         }
     } else {
