@@ -32,10 +32,11 @@ import torch
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from one ncu capture of the kernel as it stands
 # (set back to None whenever that kernel changes); the capture and its command are in the named file
 NCU_TRAFFIC = {
-    # stage 1 of cfg3: row_stream_kernel 365.5 + 108.6 MB, inplace_compact_kernel 78.5 + 27.9 MB (the plan kernel's
-    # maps are a fraction of a MB)
-    ("cfg3", "lvlm_merge_compact"): {"bytes_per_launch": 580500000,
-                                     "source": "profiles/row_stream_kernel_cfg3.txt + profiles/inplace_compact_kernel_cfg3.txt"},
+    # stage 1 of cfg3: row_stream_kernel 365.4 + 108.6 MB, inplace_compact_kernel 78.5 + 27.9 MB, merge_plan_kernel
+    # 0.25 MB
+    ("cfg3", "lvlm_merge_compact"): {"bytes_per_launch": 580700000,
+                                     "source": "profiles/row_stream_kernel_cfg3.txt + profiles/inplace_compact_kernel_cfg3.txt"
+                                               " + profiles/merge_plan_kernel_cfg3.txt"},
 }
 DOMINANT_KERNEL = {"lvlm_decode_attn": "decode_cluster_kernel", "lvlm_score_tokens": "score_tc_kernel<0> + <1>",
                    "lvlm_merge_compact": "row_stream_kernel (with merge_plan_kernel before and inplace_compact_kernel after it)",
