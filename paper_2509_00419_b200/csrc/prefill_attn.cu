@@ -3,8 +3,9 @@
 // attention kernel that runs anyway, so no separate pass over Q K^T is paid for the row normalisers).
 //
 // One CTA per (sequence, query head, tile of 128 query rows); tcgen05 MMAs, accumulators in tensor memory:
-//   S = Q K_j^T      A = Q tile, B = K tile, both K-major from TMA (128-byte swizzle), 128x128 fp32 in TMEM (two
-//                    buffers: the tile after next is multiplied while this one is in the softmax)
+//   S = Q K_j^T      A = Q tile, copied once from shared into tensor memory (bf16 pairs a column), B = K tile, K-major
+//                    from TMA (128-byte swizzle), 128x128 fp32 in TMEM (two buffers: the tile after next is multiplied
+//                    while this one is in the softmax)
 //   softmax          eight warps: thread = (query row, half of the tile's 128 keys); the row maximum of a tile meets
 //                    in shared memory (one named barrier a tile); running max m and sum l in the log2 domain.  The
 //                    probabilities 2^(s - m) go back into the tensor-memory columns the logits came from, as
@@ -33,7 +34,7 @@ constexpr int kATile = 2 * kAHalf;           // 32 KB
 constexpr int kAStages = 2;                  // K ring and V ring (released separately: K after S, V after O)
 constexpr int kASoftmaxThreads = 256;        // warps 2..9
 constexpr int kAThreads = 64 + kASoftmaxThreads;   // warp 0 TMA, warp 1 MMA
-constexpr uint32_t kATmemCols = 512;         // S0/P0 | S1/P1 | O | (unused)
+constexpr uint32_t kATmemCols = 512;         // S0/P0 | S1/P1 | O | Q (64 columns) | (unused)
 constexpr float kLog2eA = 1.4426950408889634f;
 constexpr float kLn2A = 0.6931471805599453f;
 constexpr float kRescaleStep = 8.0f;         // the output is rescaled when the row maximum has grown by more (log2)
@@ -48,7 +49,7 @@ struct AttnArgs {
 };
 
 struct AttnSmem {
-    uint64_t q_full, k_full[kAStages], k_empty[kAStages], v_full[kAStages], v_empty[kAStages], s_full[2], p_ready, o_done;
+    uint64_t q_full, k_full[kAStages], k_empty[kAStages], v_full[kAStages], v_empty[kAStages], s_full[2], p_ready, o_done, q_ready;
     uint32_t tmem_base;
     volatile int abort;
     float xmax[2][2][kAT];     // [tile parity][half][row]: the tile maximum of a half row, for the other half
@@ -134,6 +135,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
         for (int s = 0; s < 2; ++s) mbar_init(&sm->s_full[s], 1);
         mbar_init(&sm->p_ready, kASoftmaxThreads);
         mbar_init(&sm->o_done, 1);
+        mbar_init(&sm->q_ready, kAT);
         sm->abort = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -147,6 +149,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
     const uint32_t tmem_o = tmem_base + 2 * kAT;
+    const uint32_t tmem_q = tmem_base + 3 * kAT;
     pdl_enter();
 
     if (warp == 0) {
@@ -172,39 +175,45 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc_qk = idesc_bf16_f32(kAT, kAT);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kAT, kAT) | (1u << 16);     // B (the V tile) is MN-major
-            const uint32_t q_addr = smem_u32(sQ);
             // S_j into buffer j & 1, over P_{j-2} (the caller has waited for the product that read it)
+            // (this thread shares its scheduler with two softmax warps: whatever an MMA needs is worked out before the
+            // wait, so that the MMAs themselves go out back to back)
             auto issue_qk = [&](int j) -> bool {
                 const int st = j % kAStages;
-                if (!attn_wait(&sm->k_full[st], (j / kAStages) & 1, sm, a.dev_status)) return false;
-                tc_fence_after();
                 const uint32_t k_addr = smem_u32(sK + st * kATile);
                 const uint32_t d_tmem = tmem_base + (j & 1) * kAT;
+                uint64_t kd[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint32_t off = (k >> 2) * kAHalf + (k & 3) * 32;
-                    mma_bf16_ss(d_tmem, smem_desc_sw128(q_addr + off), smem_desc_sw128(k_addr + off), idesc_qk, k > 0);
-                }
+                for (int k = 0; k < 8; ++k) kd[k] = smem_desc_sw128(k_addr + (k >> 2) * kAHalf + (k & 3) * 32);
+                if (!attn_wait(&sm->k_full[st], (j / kAStages) & 1, sm, a.dev_status)) return false;
+                tc_fence_after();
+                mma_bf16_ts(d_tmem, tmem_q, kd[0], idesc_qk, 0u);       // 16 channels per step: 8 columns of bf16 pairs
+#pragma unroll
+                for (int k = 1; k < 8; ++k) mma_bf16_ts(d_tmem, tmem_q + k * 8, kd[k], idesc_qk, 1u);
                 mma_commit(&sm->k_empty[st]);              // the K tile may be refilled once these are done
                 mma_commit(&sm->s_full[j & 1]);
                 return true;
             };
-            bool ok = attn_wait(&sm->q_full, 0, sm, a.dev_status);
+            bool ok = attn_wait(&sm->q_ready, 0, sm, a.dev_status);
             if (ok && nk > 0) ok = issue_qk(0);
             if (ok && nk > 1) ok = issue_qk(1);
             for (int j = 0; ok && j < nk; ++j) {
-                ok = attn_wait(&sm->p_ready, j & 1, sm, a.dev_status);
-                if (ok) ok = attn_wait(&sm->v_full[j % kAStages], (j / kAStages) & 1, sm, a.dev_status);
-                if (!ok) break;
-                tc_fence_after();
                 const uint32_t v_addr = smem_u32(sV + (j % kAStages) * kATile);
                 const uint32_t p_tmem = tmem_base + (j & 1) * kAT;
+                uint64_t vd[8];                             // 16 keys per step: 8 columns of bf16 pairs
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {               // 16 keys per step: 8 columns of bf16 pairs
-                    const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;       // heads; the remainders lie 16 columns on
-                    const uint64_t vdesc = smem_desc_mn_sw128(v_addr + k * 2048, kAHalf);
-                    mma_bf16_ts(tmem_o, pa, vdesc, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
-                    mma_bf16_ts(tmem_o, pa + 16, vdesc, idesc_pv, 1u);
+                for (int k = 0; k < 8; ++k) vd[k] = smem_desc_mn_sw128(v_addr + k * 2048, kAHalf);
+                ok = attn_wait(&sm->v_full[j % kAStages], (j / kAStages) & 1, sm, a.dev_status);
+                if (ok) ok = attn_wait(&sm->p_ready, j & 1, sm, a.dev_status);
+                if (!ok) break;
+                tc_fence_after();
+                mma_bf16_ts(tmem_o, p_tmem, vd[0], idesc_pv, j > 0 ? 1u : 0u);       // heads; the remainders lie 16 columns on
+                mma_bf16_ts(tmem_o, p_tmem + 16, vd[0], idesc_pv, 1u);
+#pragma unroll
+                for (int k = 1; k < 8; ++k) {
+                    const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
+                    mma_bf16_ts(tmem_o, pa, vd[k], idesc_pv, 1u);
+                    mma_bf16_ts(tmem_o, pa + 16, vd[k], idesc_pv, 1u);
                 }
                 mma_commit(&sm->v_empty[j % kAStages]);     // the V tile is done with
                 mma_commit(&sm->o_done);
@@ -223,6 +232,26 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
         const int pos = qt * kAT + row;                      // sequence position of my query
         const uint32_t lane_addr = ((uint32_t)(quarter * 32) << 16);
         float m_used = -INFINITY, l_run = 0.f;               // l_run: the sum over my half of the keys
+        // The Q tile goes from shared memory into tensor memory once (thread = row, bf16 pairs a column): S = Q K^T
+        // then reads only K from shared memory, which is what lets these MMAs run at the pace of the pipe.
+        if (half == 0) {
+            const bool got = __all_sync(0xFFFFFFFFu, attn_wait(&sm->q_full, 0, sm, a.dev_status));
+            if (got) {
+#pragma unroll
+                for (int hq = 0; hq < 2; ++hq) {             // 64 channels = 32 columns
+                    uint32_t w[32];
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(sQ + hq * kAHalf + row * 128 + ((ch ^ (row & 7)) << 4));
+                        w[4 * ch] = x.x; w[4 * ch + 1] = x.y; w[4 * ch + 2] = x.z; w[4 * ch + 3] = x.w;
+                    }
+                    tmem_st32(tmem_q + lane_addr + hq * 32, reinterpret_cast<const float*>(w));
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&sm->q_ready);
+            }
+        }
         // Every thread runs every round and meets the others at the named barrier, also after a wait has given up
         // (`ok`, the same for all lanes of a warp, then only switches the work off).
         bool ok = true;
