@@ -100,6 +100,13 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
 __device__ __forceinline__ bool attn_wait(uint64_t* bar, uint32_t parity, AttnSmem* sm, int32_t* dev_status) {
     if (sm->abort) return false;
     if (mbar_wait(bar, parity)) return true;
@@ -172,7 +179,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // The whole warp runs the loop (same values in every lane, so that they can live in uniform registers); one
+        // elected lane issues the MMAs and the commits.
+        {
             constexpr uint32_t idesc_qk = idesc_bf16_f32(kAT, kAT);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kAT, kAT) | (1u << 16);     // B (the V tile) is MN-major
             // S_j into buffer j & 1, over P_{j-2} (the caller has waited for the product that read it)
@@ -185,16 +194,19 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
                 uint64_t kd[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) kd[k] = smem_desc_sw128(k_addr + (k >> 2) * kAHalf + (k & 3) * 32);
-                if (!attn_wait(&sm->k_full[st], (j / kAStages) & 1, sm, a.dev_status)) return false;
+                if (!__all_sync(0xFFFFFFFFu, attn_wait(&sm->k_full[st], (j / kAStages) & 1, sm, a.dev_status))) return false;
                 tc_fence_after();
-                mma_bf16_ts(d_tmem, tmem_q, kd[0], idesc_qk, 0u);       // 16 channels per step: 8 columns of bf16 pairs
+                if (elect_one()) {
+                    mma_bf16_ts(d_tmem, tmem_q, kd[0], idesc_qk, 0u);       // 16 channels per step: 8 columns of bf16 pairs
 #pragma unroll
-                for (int k = 1; k < 8; ++k) mma_bf16_ts(d_tmem, tmem_q + k * 8, kd[k], idesc_qk, 1u);
-                mma_commit(&sm->k_empty[st]);              // the K tile may be refilled once these are done
-                mma_commit(&sm->s_full[j & 1]);
+                    for (int k = 1; k < 8; ++k) mma_bf16_ts(d_tmem, tmem_q + k * 8, kd[k], idesc_qk, 1u);
+                    mma_commit(&sm->k_empty[st]);              // the K tile may be refilled once these are done
+                    mma_commit(&sm->s_full[j & 1]);
+                }
+                __syncwarp();
                 return true;
             };
-            bool ok = attn_wait(&sm->q_ready, 0, sm, a.dev_status);
+            bool ok = __all_sync(0xFFFFFFFFu, attn_wait(&sm->q_ready, 0, sm, a.dev_status));
             if (ok && nk > 0) ok = issue_qk(0);
             if (ok && nk > 1) ok = issue_qk(1);
             for (int j = 0; ok && j < nk; ++j) {
@@ -205,22 +217,26 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_const
                 for (int k = 0; k < 8; ++k) vd[k] = smem_desc_mn_sw128(v_addr + k * 2048, kAHalf);
                 ok = attn_wait(&sm->v_full[j % kAStages], (j / kAStages) & 1, sm, a.dev_status);
                 if (ok) ok = attn_wait(&sm->p_ready, j & 1, sm, a.dev_status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                mma_bf16_ts(tmem_o, p_tmem, vd[0], idesc_pv, j > 0 ? 1u : 0u);       // heads; the remainders lie 16 columns on
-                mma_bf16_ts(tmem_o, p_tmem + 16, vd[0], idesc_pv, 1u);
+                if (elect_one()) {
+                    mma_bf16_ts(tmem_o, p_tmem, vd[0], idesc_pv, j > 0 ? 1u : 0u);       // heads; the remainders lie 16 columns on
+                    mma_bf16_ts(tmem_o, p_tmem + 16, vd[0], idesc_pv, 1u);
 #pragma unroll
-                for (int k = 1; k < 8; ++k) {
-                    const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
-                    mma_bf16_ts(tmem_o, pa, vd[k], idesc_pv, 1u);
-                    mma_bf16_ts(tmem_o, pa + 16, vd[k], idesc_pv, 1u);
+                    for (int k = 1; k < 8; ++k) {
+                        const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
+                        mma_bf16_ts(tmem_o, pa, vd[k], idesc_pv, 1u);
+                        mma_bf16_ts(tmem_o, pa + 16, vd[k], idesc_pv, 1u);
+                    }
+                    mma_commit(&sm->v_empty[j % kAStages]);     // the V tile is done with
+                    mma_commit(&sm->o_done);
                 }
-                mma_commit(&sm->v_empty[j % kAStages]);     // the V tile is done with
-                mma_commit(&sm->o_done);
+                __syncwarp();
                 if (j + 2 < nk) {
                     // The logits of the tile after next go where this tile's P lies: not before the product has read it
                     // (the softmax of the next tile is far from done by then, so nothing waits for this wait).
-                    ok = attn_wait(&sm->o_done, j & 1, sm, a.dev_status);
+                    ok = __all_sync(0xFFFFFFFFu, attn_wait(&sm->o_done, j & 1, sm, a.dev_status));
                     if (ok) ok = issue_qk(j + 2);
                 }
             }
