@@ -439,28 +439,34 @@ nk_sim_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        // all lanes run the loop (uniform operands), one elected lane issues
+        {
             constexpr uint32_t idesc = idesc_bf16_f32(kSimM, kSimN);
             int it = 0;
             bool ok = true;
             for (int j = 0; ok && j < ntile; ++j) {
                 const int buf = j & 1;
-                if (j >= 2) ok = sim_wait(&sm->tmem_empty[buf], ((j / 2) - 1) & 1, sm, a.dev_status);
+                if (j >= 2) ok = __all_sync(0xFFFFFFFFu, sim_wait(&sm->tmem_empty[buf], ((j / 2) - 1) & 1, sm, a.dev_status));
                 for (int kc = 0; ok && kc < a.nkc; ++kc, ++it) {
                     const int st = it % kSimStages;
-                    ok = sim_wait(&sm->full[st], (it / kSimStages) & 1, sm, a.dev_status);
-                    if (!ok) break;
-                    tc_fence_after();
                     const uint32_t a_addr = smem_u32(base + st * kSimStageBytes);
                     const uint32_t b_addr = a_addr + kSimABytes;
                     const uint32_t d_tmem = tmem_base + buf * kSimN;
+                    uint64_t ad[4], bd[4];
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_bf16_ss(d_tmem, smem_desc_sw128(a_addr + kk * 32), smem_desc_sw128(b_addr + kk * 32),
-                                    idesc, (kc > 0 || kk > 0) ? 1u : 0u);
-                    mma_commit(&sm->empty[st]);
+                    for (int kk = 0; kk < 4; ++kk) { ad[kk] = smem_desc_sw128(a_addr + kk * 32); bd[kk] = smem_desc_sw128(b_addr + kk * 32); }
+                    ok = __all_sync(0xFFFFFFFFu, sim_wait(&sm->full[st], (it / kSimStages) & 1, sm, a.dev_status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(d_tmem, ad[kk], bd[kk], idesc, (kc > 0 || kk > 0) ? 1u : 0u);
+                        mma_commit(&sm->empty[st]);
+                    }
+                    __syncwarp();
                 }
-                if (ok) mma_commit(&sm->tmem_full[buf]);
+                if (ok && elect_one()) mma_commit(&sm->tmem_full[buf]);
+                __syncwarp();
             }
         }
     } else {

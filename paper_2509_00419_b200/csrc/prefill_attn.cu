@@ -100,13 +100,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// True in exactly one lane of the (converged) warp.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
-    return pred != 0;
-}
-
 __device__ __forceinline__ bool attn_wait(uint64_t* bar, uint32_t parity, AttnSmem* sm, int32_t* dev_status) {
     if (sm->abort) return false;
     if (mbar_wait(bar, parity)) return true;

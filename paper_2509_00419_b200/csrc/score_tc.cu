@@ -220,26 +220,34 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0 && nt > 0) {
+        // all lanes run the loop (uniform operands), one elected lane issues
+        if (nt > 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(kTile, kTile);
             const uint32_t a_addr = smem_u32(sA);
-            bool ok = wait_or_abort(&sm->a_full, 0, sm, a.dev_status);
+            uint64_t ad[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) ad[k] = smem_desc_sw128(a_addr + (k >> 2) * kHalfBytes + (k & 3) * 32);
+            bool ok = __all_sync(0xFFFFFFFFu, wait_or_abort(&sm->a_full, 0, sm, a.dev_status));
             for (int t = 0; ok && t < nt; ++t) {
                 const int st = t % kStages, buf = t & 1;
-                ok = wait_or_abort(&sm->full[st], (t / kStages) & 1, sm, a.dev_status);
-                if (ok && t >= 2) ok = wait_or_abort(&sm->tmem_empty[buf], ((t / 2) - 1) & 1, sm, a.dev_status);
-                if (!ok) break;
-                tc_fence_after();
                 const uint32_t b_addr = smem_u32(sB + st * kTileBytes);
                 const uint32_t d_tmem = tmem_base + buf * kTile;
+                uint64_t bd[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-                    mma_bf16_ss(d_tmem, smem_desc_sw128(a_addr + off), smem_desc_sw128(b_addr + off),
-                                idesc, k > 0);
+                for (int k = 0; k < 8; ++k) bd[k] = smem_desc_sw128(b_addr + (k >> 2) * kHalfBytes + (k & 3) * 32);
+                ok = wait_or_abort(&sm->full[st], (t / kStages) & 1, sm, a.dev_status);
+                if (ok && t >= 2) ok = wait_or_abort(&sm->tmem_empty[buf], ((t / 2) - 1) & 1, sm, a.dev_status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (elect_one()) {
+                    mma_bf16_ss(d_tmem, ad[0], bd[0], idesc, 0u);
+#pragma unroll
+                    for (int k = 1; k < 8; ++k) mma_bf16_ss(d_tmem, ad[k], bd[k], idesc, 1u);
+                    mma_commit(&sm->empty[st]);        // the stage may be refilled once these MMAs are done
+                    mma_commit(&sm->tmem_full[buf]);   // ... and the accumulator may be drained
                 }
-                mma_commit(&sm->empty[st]);        // the stage may be refilled once these MMAs are done
-                mma_commit(&sm->tmem_full[buf]);   // ... and the accumulator may be drained
+                __syncwarp();
             }
         }
     } else {
