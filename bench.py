@@ -230,11 +230,21 @@ def bench_prefill_attn(w, device, steps, warmup, flush, peaks):
     def attn_only():
         L.prefill_attn(q, k, v, N=w.N, out=out, lse=lse)
 
-    t = {}
-    for name, fn in (("attention_only", attn_only), ("attention_then_score_tokens", separate), ("fused", fused)):
-        g = P.capture(fn)
-        t[name], _ = timed(g.replay, steps, warmup, flush)
-        del g
+    # the three variants take turns inside every round, so that drift of the clock under a seconds-long run of a
+    # compute-bound kernel is shared by them (the cost of the scores is a difference of two of these times)
+    variants = (("attention_only", attn_only), ("attention_then_score_tokens", separate), ("fused", fused))
+    graphs = {name: P.capture(fn) for name, fn in variants}
+    samples = {name: [] for name, _ in variants}
+    for it in range(warmup + steps):
+        for name, _ in variants:
+            flush()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graphs[name].replay(); e1.record()
+            e1.synchronize()
+            if it >= warmup:
+                samples[name].append(e0.elapsed_time(e1))
+    t = {name: float(np.mean(v)) for name, v in samples.items()}
+    del graphs
     flops = 4.0 * w.B * w.H * 128 * (w.N * (w.N + 1) / 2)          # causal: Q K^T and P V
     return {"ms": t, "attention_tflops": flops / (t["attention_only"] * 1e9),
             "attention_frac_tensor": flops / (t["attention_only"] * 1e9) / peaks["bf16_tflops"],
